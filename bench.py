@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of batched plan evaluation: one step = one pe_eval_batch over a resident batch.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is operator-evaluations per second (candidates x
+operators / time) over all GPUs, with `plans_per_s` beside it; `roofline` rates the evaluation
+kernel against the HBM copy peak on the bytes the method must move; `e2e` is the same metric
+through the host-buffer entry point, copies included; `cpu_baseline` is the CPU oracle on a
+bounded sample of the same workload.
+"""
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2503_09357_b200 import workloads as wl  # noqa: E402
+
+WORKLOADS = {
+    "tiny_pipeline": lambda: wl.make_config(1),
+    "bidirectional_pipeline": lambda: wl.make_config(2),
+    "moe_branchy": lambda: wl.make_config(3),
+    "multimodal_mimo": lambda: wl.make_config(4),
+}
+for _V, _D in wl.SWEEP_POINTS:
+    WORKLOADS[f"random_layered_V{_V}_D{_D}"] = (lambda V=_V, D=_D: wl.make_config(5, V=V, D=D))
+DEFAULT_WORKLOAD = "random_layered_V16384_D64"   # the largest configuration: sweep point V=16384, D=64, K=65536
+
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per operator-evaluation of the
+# evaluation kernel from an ncu capture, keyed by kernel variant, valid only for the kernel
+# source whose hash is recorded with it.  Reported as null when the source has changed.
+NCU_TRAFFIC = {
+    # variant: (sha256 of csrc/pe_eval.cu at capture time, bytes per op-eval, captured workload)
+}
+
+
+def kernel_source_hash():
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2503_09357_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def compulsory_bytes(V, D, K, order_bytes, want_times=True):
+    """Bytes the method must move per launch: machine id + order entry (+ start + finish) per
+    operator-evaluation, makespan + status + busy[D] + peak[D] per candidate."""
+    per_op = 1 + order_bytes + (8 if want_times else 0)
+    return K * V * per_op + K * (8 + 8 * D)
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle samples every 100 ms; `stop(t0, t1)` keeps those taken inside the
+    wall-clock window of the timed region (or the nearest ones when the region is shorter than a period)."""
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(gpu_index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            pass
+
+    def stop(self, t0, t1):
+        import datetime
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            text, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            text, _ = self.proc.communicate()
+        rows = []
+        for line in text.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(f[1]), float(f[2]), float(f[3]), [v.lower().startswith("active") for v in f[5:9]]))
+            except ValueError:
+                continue
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        inside = [r for r in rows if t0 <= r[0] <= t1]
+        if not inside:                                    # region shorter than a sampling period: nearest sample
+            inside = [min(rows, key=lambda r: abs(r[0] - 0.5 * (t0 + t1)))]
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        reasons = sorted({n for r in inside for n, on in zip(names, r[4]) if on})
+        return {"sm_mhz": statistics.median(r[1] for r in inside), "sm_max_mhz": max(r[2] for r in inside),
+                "power_w_max": max(r[3] for r in inside), "samples": len(inside), "reasons": reasons}
+
+
+def time_oracle(w, assign, order, target_s, threads):
+    """Oracle (as it stands) on a bounded sample of the workload's candidates, ~target_s of wall time."""
+    from oracle import pe_oracle as orc
+    V, K = order.shape
+    probe = min(K, max(threads * 4, 64))
+    t0 = time.perf_counter()
+    orc.evaluate(w, np.ascontiguousarray(assign[:, :probe]), np.ascontiguousarray(order[:, :probe]), threads=threads)
+    dt = max(time.perf_counter() - t0, 1e-6)
+    n = int(min(K, max(probe, probe * target_s / dt)))
+    a = np.ascontiguousarray(assign[:, :n]); o = np.ascontiguousarray(order[:, :n])
+    t0 = time.perf_counter()
+    orc.evaluate(w, a, o, threads=threads)
+    dt = time.perf_counter() - t0
+    return n, dt
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = WORKLOADS[args.workload]()
+    V, D = w.num_ops, w.num_devices
+    threads = os.cpu_count() or 1
+    budget_s = 90.0                                          # whole run, warm-up included
+    per_step = budget_s / (args.steps + args.warmup)
+    K_gen = int(min(w.num_candidates, 8192))
+    assign, order = wl.make_candidates(w, K=K_gen)
+    n, dt = time_oracle(w, assign, order, min(per_step, 10.0) * 0.8, threads)   # sizes the per-step sample
+    if n > K_gen:
+        n = K_gen
+    from oracle import pe_oracle as orc
+    a = np.ascontiguousarray(assign[:, :n]); o = np.ascontiguousarray(order[:, :n])
+    for _ in range(args.warmup):
+        orc.evaluate(w, a, o, threads=threads)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        orc.evaluate(w, a, o, threads=threads)
+    dt = time.perf_counter() - t0
+    value = n * V * args.steps / dt
+    line = {
+        "impl": "reference", "metric": "op_evals_per_s", "value": value, "unit": "op-evals/s",
+        "plans_per_s": value / V, "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32", "data": "synthetic",
+        "config": {"workload": args.workload, "V": V, "D": D, "E": w.num_edges, "K": w.num_candidates,
+                   "outputs": "full", "sample": f"{n} candidates per step"},
+        "cpu_baseline": {"value": value, "unit": "op-evals/s", "cores": threads, "kind": "oracle",
+                         "sample": f"{n} of {w.num_candidates} candidates per step, {args.steps} steps"},
+        "e2e": {"value": value, "unit": "op-evals/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2503_09357_b200 import binding as pe
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    w = WORKLOADS[args.workload]()
+    V, D, K = w.num_ops, w.num_devices, (args.candidates or w.num_candidates)
+    want_times = args.outputs == "full"
+    flags = 0
+    obytes = 2 if V <= 65536 else 4
+    odt = torch.int16 if obytes == 2 else torch.int32
+
+    # inputs in pinned host memory (weak scaling: every rank draws its own K candidates)
+    t_gen = time.perf_counter()
+    h_assign = torch.empty((V, K), dtype=torch.uint8).pin_memory()
+    h_order = torch.empty((V, K), dtype=odt).pin_memory()
+    wl.make_candidates(w, K=K, first=rank * K, out_assign=h_assign.numpy(),
+                       out_order=h_order.numpy().view(np.uint16 if obytes == 2 else np.uint32))
+    t_gen = time.perf_counter() - t_gen
+
+    g = pe.Graph(w, device=local_rank)
+    variant = g.variant(K, flags)
+    d_assign = h_assign.to(dev, non_blocking=True)
+    d_order = h_order.to(dev, non_blocking=True)
+    d_out = g.alloc_outputs(K, want_times)
+    ws, ws_bytes = g.alloc_workspace(K, flags)
+    outs = pe.make_outputs(**{k: v.data_ptr() for k, v in d_out.items()})
+    stream = torch.cuda.current_stream(dev)
+
+    def step():
+        rc = pe.pe_eval_batch(g.handle, K, d_assign.data_ptr(), d_order.data_ptr(), obytes, flags, outs,
+                              ws.data_ptr(), ws_bytes, stream.cuda_stream)
+        if rc != pe.PE_OK:
+            raise pe.PeError(rc, "pe_eval_batch")
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    torch.cuda.synchronize(dev)
+    t_w = time.perf_counter()
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize(dev)
+    t_w = (time.perf_counter() - t_w) / args.warmup
+    if args.steps <= 0:                                     # default: about two seconds of timed work
+        args.steps = int(min(2000, max(10, 2.0 / max(t_w, 1e-5))))
+        if world > 1:
+            st = torch.tensor([args.steps], dtype=torch.int64, device=dev)
+            dist.all_reduce(st, op=dist.ReduceOp.MAX)
+            args.steps = int(st.item())
+
+    # ---- timed region: device resident, CUDA events on the launching stream ----
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches0 = pe.pe_kernel_launches()
+    barrier(); torch.cuda.synchronize(dev)
+    t_first = torch.cuda.Event(enable_timing=True); t_last = torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
+    t_first.record(stream)
+    for a, b in ev:
+        a.record(stream); step(); b.record(stream)
+    t_last.record(stream)
+    torch.cuda.synchronize(dev)
+    wall1 = time.time()
+    barrier()
+    launches = pe.pe_kernel_launches() - launches0
+    clocks = sampler.stop(wall0, wall1) if sampler else None
+    total_ms = t_first.elapsed_time(t_last)
+    kernel_ms = [a.elapsed_time(b) for a, b in ev]
+    if pe.pe_graph_poll_error(g.handle, stream.cuda_stream) != pe.PE_OK:
+        raise SystemExit("device-side error word set during the timed region")
+    tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    value = world * K * V / (ms_per_step * 1e-3)
+
+    # ---- end to end: host buffers through pe_eval_batch_host, copies inside the timed region ----
+    h_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in d_out.items()}
+    houts = pe.make_outputs(**{k: v.data_ptr() for k, v in h_out.items()})
+
+    def e2e_step():
+        rc = pe.pe_eval_batch_host(g.handle, K, h_assign.data_ptr(), h_order.data_ptr(), obytes, flags, houts,
+                                   d_assign.data_ptr(), d_order.data_ptr(), outs, ws.data_ptr(), ws_bytes,
+                                   stream.cuda_stream)
+        if rc != pe.PE_OK:
+            raise pe.PeError(rc, "pe_eval_batch_host")
+
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    e2e_step()
+    barrier(); torch.cuda.synchronize(dev)
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    torch.cuda.synchronize(dev)
+    e2e_s = time.perf_counter() - t0
+    te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_value = world * K * V * e2e_steps / float(te.item())
+    h2d = V * K * (1 + obytes)
+    d2h = sum(v.numel() * v.element_size() for v in d_out.values())
+
+    if rank == 0:
+        peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        if os.path.exists(peaks_path):
+            peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+        else:
+            peak, peak_src = FALLBACK_HBM_GBS, "fallback"
+        kms = statistics.mean(kernel_ms)
+        alg = compulsory_bytes(V, D, K, obytes, want_times)
+        achieved = alg / (kms * 1e-3) / 1e9
+        traffic = None
+        rec = NCU_TRAFFIC.get(variant)
+        if rec and rec[0] == kernel_source_hash():
+            traffic = rec[1] * K * V
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            threads = os.cpu_count() or 1
+            n, dt = time_oracle(w, h_assign.numpy(), h_order.numpy().view(np.uint16 if obytes == 2 else np.uint32),
+                                args.cpu_seconds, threads)
+            cpu = {"value": n * V / dt, "unit": "op-evals/s", "cores": threads, "kind": "oracle",
+                   "sample": f"first {n} of {K} candidates, all outputs, {dt:.1f} s"}
+        line = {
+            "metric": "op_evals_per_s", "value": value, "unit": "op-evals/s", "plans_per_s": value / V,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+            "config": {"workload": args.workload, "V": V, "E": w.num_edges, "D": D, "L": w.num_link_classes,
+                       "K_per_gpu": K, "outputs": args.outputs, "order_bytes": obytes, "kernel_variant": variant,
+                       "l2": "inputs and outputs larger than L2" if alg > 252e6 else "working set below 2x L2: not flushed",
+                       "candidate_generation_s": round(t_gen, 1)},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": traffic, "peak_source": f"of {peak_src}", "kernel": f"pe_eval_{variant}_kernel",
+                         "kernel_ms": kms, "algorithmic_bytes_per_launch": alg},
+            "e2e": {"value": e2e_value, "unit": "op-evals/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps},
+            "gpu_launches": launches, "clocks": clocks, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    g.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=0, help="timed steps (default: enough for about 2 s)")
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default=DEFAULT_WORKLOAD)
+    ap.add_argument("--outputs", choices=["full", "summary"], default="full")
+    ap.add_argument("--candidates", type=int, default=0, help="override K per GPU (default: the configuration's K)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        args.steps = args.steps if args.steps > 0 else 5
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

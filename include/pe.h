@@ -1,0 +1,150 @@
+/* pe.h — batched evaluation of candidate parallel plans (C ABI).
+ *
+ * Problem data follow the problem statement of Section III of "Automatic Operator-level
+ * Parallelism Planning for Distributed Deep Learning — A Mixed-Integer Programming
+ * Approach" (arXiv 2503.09357): an operator DAG G_m(I, B) with durations D^o_i, per-edge
+ * communication durations D^c, memory adjustments A_i and weights W_i, and a cluster of
+ * machines whose channels are grouped into link classes, each machine with a memory limit.
+ *
+ * A candidate plan is (x, pi): x[i] is the machine of operator i (Eq. 6) and pi a global
+ * priority order that is a topological order of G_m; pi fixes every precedence variable
+ * y of Eqs. 7-8.  For each candidate the library computes the componentwise-least start
+ * and end times satisfying Eq. 3, Eqs. 7-8 and Eqs. 11-13 (communication is a delay
+ * charged only between different machines), the makespan (Eqs. 1-2), each machine's busy
+ * time (its bubble is makespan - busy) and each machine's peak memory level along its own
+ * operator sequence (Eqs. 16-19), plus status flags.  All quantities are int32.
+ *
+ * Layout.  Per-candidate arrays are candidate-interleaved: element (row, c) of an [R][K]
+ * array is at index row*K + c.  "By-op" arrays have one row per operator id, "by-pos"
+ * arrays one row per position k of the priority order, per-machine arrays one row per
+ * machine.
+ *
+ * Threading / ownership.  A pe_graph is immutable after creation and may be used from
+ * several host threads and streams.  The library allocates device memory only in
+ * pe_graph_create (the graph copy, a few KB..MB); candidates, outputs and workspace
+ * belong to the caller.  No function throws; every error is a negative return code.
+ */
+#ifndef PE_H_
+#define PE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pe_graph pe_graph; /* opaque; owns the device copy of the problem data */
+
+/* Return codes. */
+enum {
+  PE_OK = 0,
+  PE_ERR_INVALID_ARG = -1, /* NULL where data is required, sizes out of range, bad flags */
+  PE_ERR_CYCLE = -2,       /* the edge list is not a DAG */
+  PE_ERR_RANGE = -3,       /* negative duration / communication / weight, edge endpoint or link class out of range */
+  PE_ERR_OVERFLOW = -4,    /* sum(dur) + sum_e max_l comm, or sum|A| + sum W, does not fit in int32 */
+  PE_ERR_CUDA = -5,        /* a CUDA runtime call failed (no device, out of memory, launch error) */
+  PE_ERR_WORKSPACE = -6,   /* workspace pointer NULL or smaller than pe_workspace_bytes() */
+  PE_ERR_TIMEOUT = -7,     /* a bounded device-side wait expired (reported by pe_graph_poll_error) */
+  PE_ERR_UNSUPPORTED = -8  /* the requested kernel variant cannot run this problem size */
+};
+
+/* Problem data (Section III).  All pointers are HOST pointers, read during the call only. */
+typedef struct {
+  int32_t num_ops;             /* V = |I| >= 1 */
+  int32_t num_edges;           /* E = |B| >= 0 */
+  const int32_t* edge_src;     /* [E] i1 of (i1, i2) in B */
+  const int32_t* edge_dst;     /* [E] i2 */
+  const int32_t* dur;          /* [V] D^o_i >= 0 */
+  const int32_t* mem_delta;    /* [V] A_i, signed; NULL = all 0 */
+  const int32_t* mem_weight;   /* [V] W_i >= 0; NULL = all 0 */
+  int32_t num_devices;         /* D = |J|, 1..255 */
+  int32_t num_link_classes;    /* L, 1..254 */
+  const uint8_t* link_class;   /* [D*D] row-major: class of the channel (machine of i1 -> machine of i2);
+                                  the diagonal is ignored; 0xFF = no channel (Eq. 10); NULL = all class 0 */
+  const int32_t* comm;         /* [E*L] D^c of edge e over link class l at e*L + l, >= 0; NULL = all 0 */
+  const int32_t* mem_capacity; /* [D] memory limit per machine; NULL = no limit */
+} pe_graph_desc;
+
+/* Host-only check of a description: ranges, acyclicity, overflow bounds.  Touches no GPU. */
+int pe_graph_validate(const pe_graph_desc* desc);
+
+/* Validate, build the by-predecessor CSR and upload it to CUDA device `cuda_device`.
+ * On success *out owns the device copy until pe_destroy.  Synchronous. */
+int pe_graph_create(const pe_graph_desc* desc, int cuda_device, pe_graph** out);
+
+/* Free the device copy.  NULL is accepted.  The caller must have finished all work using it. */
+int pe_destroy(pe_graph* g);
+
+/* Flags of pe_eval_batch. */
+enum {
+  PE_ASSIGN_BY_POS = 1u, /* `assign` row k holds x[pi[k]] (the machine sequence) instead of row i holding x[i] */
+  PE_TIMES_BY_OP = 2u,   /* `start` / `finish` row i belongs to operator i instead of row k to position k */
+  /* Kernel variant (bits 8..11); 0 lets the library choose from (V, E, D, L) and the device. */
+  PE_VARIANT_AUTO = 0u << 8,
+  PE_VARIANT_GLOBAL = 1u << 8, /* one thread per candidate, finish-time state in the caller's workspace */
+  PE_VARIANT_SHARED = 2u << 8, /* one thread per candidate, finish-time state in shared memory */
+  PE_VARIANT_WARP = 3u << 8,   /* one warp per candidate, finish-time state in shared memory */
+  PE_VARIANT_MASK = 15u << 8
+};
+
+/* Status bits per candidate (0 = a valid topological permutation, feasible). */
+enum {
+  PE_STATUS_ASSIGN_RANGE = 1u,  /* a consulted machine id is >= D */
+  PE_STATUS_ORDER_INVALID = 2u, /* an order entry >= V, a repeated operator, or an operator placed before a predecessor */
+  PE_STATUS_MEM_EXCEEDED = 4u,  /* some machine's peak memory level is above its capacity (Section III) */
+  PE_STATUS_NO_CHANNEL = 8u     /* an edge crosses a machine pair whose link class is 0xFF (Eq. 10); delay taken as 0 */
+};
+/* For a candidate with bit 1 or 2 set every other output (and status bits 4, 8) is unspecified. */
+
+/* Outputs: DEVICE pointers owned by the caller; a NULL member is not computed/written. */
+typedef struct {
+  int32_t* start;    /* [V*K] s, by-pos (default) or by-op (PE_TIMES_BY_OP) */
+  int32_t* finish;   /* [V*K] e, same layout */
+  int32_t* makespan; /* [K]   max_i e_i (Eq. 2) */
+  int32_t* busy;     /* [D*K] sum of D^o over the operators of machine j */
+  int32_t* peak_mem; /* [D*K] max over prefixes (the empty one included) of the machine's memory level */
+  uint32_t* status;  /* [K]   PE_STATUS_* bits */
+} pe_outputs;
+
+/* Bytes of device workspace pe_eval_batch needs for K candidates with these flags (may be 0). */
+size_t pe_workspace_bytes(const pe_graph* g, int64_t K, uint32_t flags);
+
+/* Which kernel variant (PE_VARIANT_*) a call with these arguments runs; negative = error code. */
+int pe_eval_variant(const pe_graph* g, int64_t K, uint32_t flags);
+
+/* Evaluate K candidates.  Asynchronous on `cuda_stream` (a cudaStream_t; NULL = default stream);
+ * never synchronises.  K = 0 is a successful no-op.
+ *   assign      device, u8 [V*K]: by-op x_c[i] at i*K + c, or by-pos under PE_ASSIGN_BY_POS
+ *   order       device, [V*K] by-pos pi_c[k] at k*K + c; uint16_t if order_bytes == 2 (V <= 65536), uint32_t if 4
+ *   out         outputs wanted (struct read during the call)
+ *   workspace   device scratch of at least pe_workspace_bytes() bytes, 256-byte aligned; contents are
+ *               overwritten; calls running concurrently must not share it
+ * Precondition: every candidate's order is a topological permutation and every machine id < D;
+ * violations are flagged per candidate in `status` and never index out of bounds. */
+int pe_eval_batch(pe_graph* g, int64_t K, const uint8_t* assign, const void* order, int order_bytes, uint32_t flags,
+                  const pe_outputs* out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Host-buffer form of the same call: copies `assign` and `order` from HOST memory into the caller's
+ * device staging buffers, evaluates, copies every requested output back to the HOST pointers in
+ * `host_out`, and synchronises the stream before returning.  `dev_assign` [V*K] u8, `dev_order`
+ * [V*K*order_bytes] and `dev_out` (device pointers for exactly the members set in host_out) are
+ * caller-owned staging.  Pinned host memory makes the copies asynchronous with each other. */
+int pe_eval_batch_host(pe_graph* g, int64_t K, const uint8_t* host_assign, const void* host_order, int order_bytes,
+                       uint32_t flags, const pe_outputs* host_out, uint8_t* dev_assign, void* dev_order,
+                       const pe_outputs* dev_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Synchronise `cuda_stream` and return the graph's device-side error word: PE_OK, or
+ * PE_ERR_TIMEOUT if a kernel gave up a bounded wait (its outputs are then invalid).  Clears the word. */
+int pe_graph_poll_error(pe_graph* g, void* cuda_stream);
+
+/* Number of kernels this library has launched in this process so far (all graphs, all streams). */
+int64_t pe_kernel_launches(void);
+
+/* Static description of an error code. */
+const char* pe_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PE_H_ */

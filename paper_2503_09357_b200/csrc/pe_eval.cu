@@ -1,0 +1,384 @@
+// pe_eval_batch: kernel variants and their dispatch.
+//
+// Every variant evaluates a candidate by one pass over its priority order (serial schedule
+// generation): at position k the operator i = pi[k] on machine j = x[i] starts at
+// max(ready time from its predecessors' end times plus cross-machine delays (Eqs. 11-13),
+// end of the previous operator on machine j (Eqs. 7-8)), ends D^o_i later (Eq. 3), and the
+// machine's memory level moves by A_i (Eqs. 16-19).  The variants differ in where the
+// per-candidate state lives and how lanes map to candidates.
+#include <atomic>
+#include <climits>
+#include <cstdio>
+
+#include "pe_device.cuh"
+#include "pe_graph.h"
+
+namespace pe {
+
+static std::atomic<int64_t> g_launches{0};
+
+// ============================================================================================
+// Variant GLOBAL: one thread per candidate; end time of every operator in the caller's
+// workspace, candidate-interleaved ([V][K] int32, -1 = not scheduled yet), machine of every
+// operator either read back from `assign` (by-op layout) or kept in a second workspace array
+// (by-position layout).  Works for any V, any time bound below 2^31, u16 or u32 orders.
+// Per-machine state (free time, level, peak, busy, weight sum) sits in shared memory,
+// [array][machine][thread] so that a warp's accesses fall in distinct banks.
+// ============================================================================================
+template <typename OrderT, bool BY_POS>
+__global__ void pe_eval_global_kernel(PeGraphView g, const uint8_t* __restrict__ blob, int64_t K,
+                                      const uint8_t* __restrict__ assign, const OrderT* __restrict__ order,
+                                      pe_outputs out, uint32_t flags, int32_t* __restrict__ e_state,
+                                      uint8_t* __restrict__ x_state) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  int32_t* dev = reinterpret_cast<int32_t*>(smem_raw);
+  const int T = blockDim.x;
+  const int t = threadIdx.x;
+  const int64_t c = (int64_t)blockIdx.x * T + t;
+  if (c >= K) return;
+  const GraphPtrs gp = graph_ptrs(blob, g);
+  const int D = g.D, V = g.V, L = g.L;
+  const size_t Ks = (size_t)K;
+  int32_t* free_at = dev + t;
+  int32_t* lvl = dev + (size_t)1 * D * T + t;
+  int32_t* peak = dev + (size_t)2 * D * T + t;
+  int32_t* busy = dev + (size_t)3 * D * T + t;
+  int32_t* wsum = dev + (size_t)4 * D * T + t;
+  for (int j = 0; j < D; ++j) {
+    free_at[j * T] = 0; lvl[j * T] = 0; peak[j * T] = 0; busy[j * T] = 0; wsum[j * T] = 0;
+  }
+  const bool by_op_times = (flags & PE_TIMES_BY_OP) != 0;
+  uint32_t st = 0;
+  int32_t z = 0;
+  for (int k = 0; k < V; ++k) {
+    const uint32_t iu = order[(size_t)k * Ks + c];
+    if (iu >= (uint32_t)V) { st |= PE_STATUS_ORDER_INVALID; continue; }
+    const int i = (int)iu;
+    uint32_t jr = BY_POS ? assign[(size_t)k * Ks + c] : assign[(size_t)i * Ks + c];
+    if (jr >= (uint32_t)D) { st |= PE_STATUS_ASSIGN_RANGE; jr = D - 1; }
+    const int j = (int)jr;
+    const PeOpRec op = load_op(gp.ops, i);
+    if (e_state[(size_t)i * Ks + c] >= 0) st |= PE_STATUS_ORDER_INVALID;
+    int32_t r = 0;
+    for (int q = op.edge_begin; q < op.edge_begin + op.indeg; ++q) {
+      const int p = gp.pred[q];
+      int32_t ep = e_state[(size_t)p * Ks + c];
+      if (ep < 0) { st |= PE_STATUS_ORDER_INVALID; continue; }
+      uint32_t xp = BY_POS ? x_state[(size_t)p * Ks + c] : assign[(size_t)p * Ks + c];
+      if (xp >= (uint32_t)D) xp = D - 1;
+      if ((int)xp != j) {
+        const uint32_t cl = gp.cls[xp * D + j];
+        if (cl == 0xFFu) st |= PE_STATUS_NO_CHANNEL;
+        else ep += gp.comm[(size_t)q * L + cl];
+      }
+      r = max(r, ep);
+    }
+    const int32_t s = max(r, free_at[j * T]);
+    const int32_t e = s + op.dur;
+    free_at[j * T] = e;
+    e_state[(size_t)i * Ks + c] = e;
+    if (BY_POS) x_state[(size_t)i * Ks + c] = (uint8_t)j;
+    busy[j * T] += op.dur;
+    const int32_t lv = lvl[j * T] + op.mem_delta;
+    lvl[j * T] = lv;
+    peak[j * T] = max(peak[j * T], lv);
+    if (gp.weight) wsum[j * T] += gp.weight[i];
+    z = max(z, e);
+    const size_t at = (size_t)(by_op_times ? i : k) * Ks + c;
+    if (out.start) out.start[at] = s;
+    if (out.finish) out.finish[at] = e;
+  }
+  for (int j = 0; j < D; ++j) {
+    const int32_t pk = peak[j * T] + wsum[j * T];  // the weights are resident from the start (Eq. 16)
+    if (pk > gp.cap[j]) st |= PE_STATUS_MEM_EXCEEDED;
+    if (out.busy) out.busy[(size_t)j * Ks + c] = busy[j * T];
+    if (out.peak_mem) out.peak_mem[(size_t)j * Ks + c] = pk;
+  }
+  if (out.makespan) out.makespan[c] = z;
+  if (out.status) out.status[c] = st;
+}
+
+// ============================================================================================
+// Variant SHARED: one thread per candidate; the per-operator state (end time and machine,
+// packed in one 32-bit word) lives in shared memory as [operator][thread], so a lane's
+// gathers stay in its own bank.  The graph blob is staged into shared memory by bulk copy
+// when it fits next to the state, otherwise read through the read-only cache.  Needs the
+// graph's time bound below 2^24 - 256.
+// ============================================================================================
+template <typename OrderT, bool BY_POS, bool GRAPH_SMEM>
+__global__ void pe_eval_shared_kernel(PeGraphView g, const uint8_t* __restrict__ blob, int64_t K,
+                                      const uint8_t* __restrict__ assign, const OrderT* __restrict__ order,
+                                      pe_outputs out, uint32_t flags, int* err) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  const int T = blockDim.x;
+  const int t = threadIdx.x;
+  const int D = g.D, V = g.V, L = g.L;
+  uint8_t* sm = smem_raw;
+  const uint8_t* gbase = blob;
+  if (GRAPH_SMEM) {
+    uint64_t* bar = reinterpret_cast<uint64_t*>(sm + g.lay.bytes);
+    if (!stage_blob(sm, blob, g.lay.bytes, bar, err)) return;
+    gbase = sm;
+    sm += g.lay.bytes + 16;
+  }
+  const GraphPtrs gp = graph_ptrs(gbase, g);
+  uint32_t* state = reinterpret_cast<uint32_t*>(sm) + t;           // [V][T]
+  int32_t* dev = reinterpret_cast<int32_t*>(sm) + (size_t)V * T + t;  // [5][D][T]
+  int32_t* free_at = dev;
+  int32_t* lvl = dev + (size_t)1 * D * T;
+  int32_t* peak = dev + (size_t)2 * D * T;
+  int32_t* busy = dev + (size_t)3 * D * T;
+  int32_t* wsum = dev + (size_t)4 * D * T;
+
+  const int64_t c = (int64_t)blockIdx.x * T + t;
+  if (c >= K) return;
+  const size_t Ks = (size_t)K;
+  for (int i = 0; i < V; ++i) state[(size_t)i * T] = 0xFFFFFFFFu;
+  for (int j = 0; j < D; ++j) {
+    free_at[j * T] = 0; lvl[j * T] = 0; peak[j * T] = 0; busy[j * T] = 0;
+    if (gp.weight) wsum[j * T] = 0;
+  }
+  const bool by_op_times = (flags & PE_TIMES_BY_OP) != 0;
+  uint32_t st = 0;
+  int32_t z = 0;
+
+  // software prefetch: order entry two positions ahead, machine id one position ahead
+  uint32_t o_cur = order[c];
+  uint32_t o_nxt = V > 1 ? (uint32_t)order[Ks + c] : 0u;
+  uint32_t a_cur = BY_POS ? assign[c] : assign[(size_t)min(o_cur, (uint32_t)(V - 1)) * Ks + c];
+  for (int k = 0; k < V; ++k) {
+    const uint32_t iu = o_cur;
+    uint32_t jr = a_cur;
+    o_cur = o_nxt;
+    if (k + 2 < V) o_nxt = order[(size_t)(k + 2) * Ks + c];
+    if (k + 1 < V) a_cur = BY_POS ? assign[(size_t)(k + 1) * Ks + c] : assign[(size_t)min(o_cur, (uint32_t)(V - 1)) * Ks + c];
+    if (iu >= (uint32_t)V) { st |= PE_STATUS_ORDER_INVALID; continue; }
+    const int i = (int)iu;
+    if (jr >= (uint32_t)D) { st |= PE_STATUS_ASSIGN_RANGE; jr = D - 1; }
+    const int j = (int)jr;
+    const PeOpRec op = load_op(gp.ops, i);
+    if (state_time(state[(size_t)i * T]) != kNotDoneTime) st |= PE_STATUS_ORDER_INVALID;
+    int32_t r = 0;
+    for (int q = op.edge_begin; q < op.edge_begin + op.indeg; ++q) {
+      const int p = gp.pred[q];
+      const uint32_t w = state[(size_t)p * T];
+      if (state_time(w) == kNotDoneTime) { st |= PE_STATUS_ORDER_INVALID; continue; }
+      int32_t ep = (int32_t)state_time(w);
+      const int xp = (int)state_dev(w);
+      if (xp != j) {
+        const uint32_t cl = gp.cls[xp * D + j];
+        if (cl == 0xFFu) st |= PE_STATUS_NO_CHANNEL;
+        else ep += gp.comm[(size_t)q * L + cl];
+      }
+      r = max(r, ep);
+    }
+    const int32_t s = max(r, free_at[j * T]);
+    const int32_t e = s + op.dur;
+    free_at[j * T] = e;
+    state[(size_t)i * T] = pack_state((uint32_t)e, (uint32_t)j);
+    busy[j * T] += op.dur;
+    const int32_t lv = lvl[j * T] + op.mem_delta;
+    lvl[j * T] = lv;
+    peak[j * T] = max(peak[j * T], lv);
+    if (gp.weight) wsum[j * T] += gp.weight[i];
+    z = max(z, e);
+    const size_t at = (size_t)(by_op_times ? i : k) * Ks + c;
+    if (out.start) out.start[at] = s;
+    if (out.finish) out.finish[at] = e;
+  }
+  for (int j = 0; j < D; ++j) {
+    const int32_t pk = peak[j * T] + (gp.weight ? wsum[j * T] : 0);
+    if (pk > gp.cap[j]) st |= PE_STATUS_MEM_EXCEEDED;
+    if (out.busy) out.busy[(size_t)j * Ks + c] = busy[j * T];
+    if (out.peak_mem) out.peak_mem[(size_t)j * Ks + c] = pk;
+  }
+  if (out.makespan) out.makespan[c] = z;
+  if (out.status) out.status[c] = st;
+}
+
+// ============================================================================================
+// Host-side planning: which variant, with what launch shape.
+// ============================================================================================
+struct Plan {
+  int variant;        // PE_VARIANT_* value
+  int threads;        // block size
+  size_t smem;        // dynamic shared memory per block
+  bool graph_smem;    // graph blob staged into shared memory
+  size_t workspace;   // bytes of caller workspace
+  size_t ws_x_off;    // offset of the machine-state array inside the workspace (GLOBAL, by-pos)
+};
+
+static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static bool plan_shared(const pe_graph* g, Plan* p) {
+  if (g->time_bound >= kPackedTimeLimit) return false;
+  const size_t per_thread = (size_t)4 * g->V + (size_t)(g->has_weight ? 20 : 16) * g->D;
+  const size_t budget = g->smem_optin;
+  for (int with_graph = 1; with_graph >= 0; --with_graph) {
+    const size_t fixed = with_graph ? (size_t)g->lay.bytes + 16 : 0;
+    if (fixed + 32 * per_thread > budget) continue;
+    size_t T = (budget - fixed) / per_thread / 32 * 32;
+    if (T > 256) T = 256;
+    p->variant = PE_VARIANT_SHARED;
+    p->threads = (int)T;
+    p->smem = fixed + T * per_thread;
+    p->graph_smem = with_graph != 0;
+    p->workspace = 0;
+    p->ws_x_off = 0;
+    return true;
+  }
+  return false;
+}
+
+static bool plan_global(const pe_graph* g, int64_t K, uint32_t flags, Plan* p) {
+  const size_t per_thread = (size_t)20 * g->D;
+  size_t T = g->smem_optin / per_thread / 32 * 32;
+  if (T > 128) T = 128;
+  if (T < 32) return false;
+  p->variant = PE_VARIANT_GLOBAL;
+  p->threads = (int)T;
+  p->smem = T * per_thread;
+  p->graph_smem = false;
+  p->ws_x_off = round_up((size_t)g->V * (size_t)K * 4, 256);
+  p->workspace = p->ws_x_off + ((flags & PE_ASSIGN_BY_POS) ? round_up((size_t)g->V * (size_t)K, 256) : 0);
+  return true;
+}
+
+static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, Plan* p) {
+  if (!g || K < 0) return PE_ERR_INVALID_ARG;
+  if (flags & ~(uint32_t)(PE_ASSIGN_BY_POS | PE_TIMES_BY_OP | PE_VARIANT_MASK)) return PE_ERR_INVALID_ARG;
+  const uint32_t want = flags & PE_VARIANT_MASK;
+  switch (want) {
+    case PE_VARIANT_AUTO:
+      if (plan_shared(g, p)) return PE_OK;
+      return plan_global(g, K, flags, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+    case PE_VARIANT_GLOBAL: return plan_global(g, K, flags, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+    case PE_VARIANT_SHARED: return plan_shared(g, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+    default: return PE_ERR_UNSUPPORTED;
+  }
+}
+
+template <typename Kern>
+static bool set_smem(Kern kern, size_t bytes) {
+  return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
+}
+
+template <typename OrderT, bool BY_POS>
+static int launch_typed(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* assign, const void* order,
+                        uint32_t flags, const pe_outputs& out, void* workspace, cudaStream_t stream) {
+  const PeGraphView view = pe_view(g);
+  const unsigned grid = (unsigned)((K + p.threads - 1) / p.threads);
+  const OrderT* ord = static_cast<const OrderT*>(order);
+  if (p.variant == PE_VARIANT_GLOBAL) {
+    int32_t* e_state = static_cast<int32_t*>(workspace);
+    uint8_t* x_state = static_cast<uint8_t*>(workspace) + p.ws_x_off;
+    if (cudaMemsetAsync(e_state, 0xFF, (size_t)g->V * (size_t)K * 4, stream) != cudaSuccess) return PE_ERR_CUDA;
+    auto kern = pe_eval_global_kernel<OrderT, BY_POS>;
+    if (!set_smem(kern, p.smem)) return PE_ERR_CUDA;
+    kern<<<grid, p.threads, p.smem, stream>>>(view, g->d_blob, K, assign, ord, out, flags, e_state, x_state);
+  } else if (p.variant == PE_VARIANT_SHARED) {
+    if (p.graph_smem) {
+      auto kern = pe_eval_shared_kernel<OrderT, BY_POS, true>;
+      if (!set_smem(kern, p.smem)) return PE_ERR_CUDA;
+      kern<<<grid, p.threads, p.smem, stream>>>(view, g->d_blob, K, assign, ord, out, flags, g->d_error);
+    } else {
+      auto kern = pe_eval_shared_kernel<OrderT, BY_POS, false>;
+      if (!set_smem(kern, p.smem)) return PE_ERR_CUDA;
+      kern<<<grid, p.threads, p.smem, stream>>>(view, g->d_blob, K, assign, ord, out, flags, g->d_error);
+    }
+  } else {
+    return PE_ERR_UNSUPPORTED;
+  }
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return cudaGetLastError() == cudaSuccess ? PE_OK : PE_ERR_CUDA;
+}
+
+}  // namespace pe
+
+extern "C" size_t pe_workspace_bytes(const pe_graph* g, int64_t K, uint32_t flags) {
+  pe::Plan p;
+  if (pe::make_plan(g, K, flags, &p) != PE_OK) return 0;
+  return p.workspace;
+}
+
+extern "C" int pe_eval_variant(const pe_graph* g, int64_t K, uint32_t flags) {
+  pe::Plan p;
+  const int rc = pe::make_plan(g, K, flags, &p);
+  return rc != PE_OK ? rc : p.variant;
+}
+
+extern "C" int64_t pe_kernel_launches(void) { return pe::g_launches.load(std::memory_order_relaxed); }
+
+extern "C" int pe_eval_batch(pe_graph* g, int64_t K, const uint8_t* assign, const void* order, int order_bytes,
+                             uint32_t flags, const pe_outputs* out, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream) {
+  if (!g || !out || K < 0) return PE_ERR_INVALID_ARG;
+  if (order_bytes != 2 && order_bytes != 4) return PE_ERR_INVALID_ARG;
+  if (order_bytes == 2 && g->V > 65536) return PE_ERR_INVALID_ARG;
+  pe::Plan p;
+  const int rc = pe::make_plan(g, K, flags, &p);
+  if (rc != PE_OK) return rc;
+  if (K == 0) return PE_OK;
+  if (!assign || !order) return PE_ERR_INVALID_ARG;
+  if ((K + p.threads - 1) / p.threads > (int64_t)INT_MAX) return PE_ERR_INVALID_ARG;
+  if (p.workspace > 0 && (!workspace || workspace_bytes < p.workspace)) return PE_ERR_WORKSPACE;
+  int prev = -1;
+  if (cudaGetDevice(&prev) != cudaSuccess) return PE_ERR_CUDA;
+  if (prev != g->device && cudaSetDevice(g->device) != cudaSuccess) return PE_ERR_CUDA;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const bool by_pos = (flags & PE_ASSIGN_BY_POS) != 0;
+  int ret;
+  if (order_bytes == 2)
+    ret = by_pos ? pe::launch_typed<uint16_t, true>(g, p, K, assign, order, flags, *out, workspace, stream)
+                 : pe::launch_typed<uint16_t, false>(g, p, K, assign, order, flags, *out, workspace, stream);
+  else
+    ret = by_pos ? pe::launch_typed<uint32_t, true>(g, p, K, assign, order, flags, *out, workspace, stream)
+                 : pe::launch_typed<uint32_t, false>(g, p, K, assign, order, flags, *out, workspace, stream);
+  if (prev != g->device) cudaSetDevice(prev);
+  return ret;
+}
+
+extern "C" int pe_eval_batch_host(pe_graph* g, int64_t K, const uint8_t* host_assign, const void* host_order,
+                                  int order_bytes, uint32_t flags, const pe_outputs* host_out, uint8_t* dev_assign,
+                                  void* dev_order, const pe_outputs* dev_out, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream) {
+  if (!g || !host_out || !dev_out || K < 0) return PE_ERR_INVALID_ARG;
+  if (order_bytes != 2 && order_bytes != 4) return PE_ERR_INVALID_ARG;
+  if (K == 0) return PE_OK;
+  if (!host_assign || !host_order || !dev_assign || !dev_order) return PE_ERR_INVALID_ARG;
+  // every output wanted on the host needs its device staging buffer
+  if ((host_out->start && !dev_out->start) || (host_out->finish && !dev_out->finish) ||
+      (host_out->makespan && !dev_out->makespan) || (host_out->busy && !dev_out->busy) ||
+      (host_out->peak_mem && !dev_out->peak_mem) || (host_out->status && !dev_out->status))
+    return PE_ERR_INVALID_ARG;
+  int prev = -1;
+  if (cudaGetDevice(&prev) != cudaSuccess) return PE_ERR_CUDA;
+  if (prev != g->device && cudaSetDevice(g->device) != cudaSuccess) return PE_ERR_CUDA;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const size_t VK = (size_t)g->V * (size_t)K, DK = (size_t)g->D * (size_t)K;
+  int ret = PE_OK;
+  if (cudaMemcpyAsync(dev_assign, host_assign, VK, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(dev_order, host_order, VK * (size_t)order_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    ret = PE_ERR_CUDA;
+  pe_outputs run = *dev_out;  // compute only what the host asked for
+  if (!host_out->start) run.start = nullptr;
+  if (!host_out->finish) run.finish = nullptr;
+  if (!host_out->makespan) run.makespan = nullptr;
+  if (!host_out->busy) run.busy = nullptr;
+  if (!host_out->peak_mem) run.peak_mem = nullptr;
+  if (!host_out->status) run.status = nullptr;
+  if (ret == PE_OK)
+    ret = pe_eval_batch(g, K, dev_assign, dev_order, order_bytes, flags, &run, workspace, workspace_bytes, cuda_stream);
+  auto back = [&](void* h, const void* d, size_t bytes) {
+    if (ret == PE_OK && h && cudaMemcpyAsync(h, d, bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) ret = PE_ERR_CUDA;
+  };
+  back(host_out->start, run.start, VK * 4);
+  back(host_out->finish, run.finish, VK * 4);
+  back(host_out->makespan, run.makespan, (size_t)K * 4);
+  back(host_out->busy, run.busy, DK * 4);
+  back(host_out->peak_mem, run.peak_mem, DK * 4);
+  back(host_out->status, run.status, (size_t)K * 4);
+  if (cudaStreamSynchronize(stream) != cudaSuccess && ret == PE_OK) ret = PE_ERR_CUDA;
+  if (prev != g->device) cudaSetDevice(prev);
+  return ret;
+}

@@ -1,0 +1,196 @@
+// Host side of the library: description checks, by-predecessor CSR, upload, teardown.
+#include <climits>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "pe_graph.h"
+
+namespace {
+
+inline uint32_t align16(uint64_t x) { return (uint32_t)((x + 15u) & ~(uint64_t)15u); }
+
+// Ranges, acyclicity and overflow bounds; fills the bounds when asked.
+int check_desc(const pe_graph_desc* d, int64_t* time_bound, int64_t* mem_bound, int32_t* max_indeg) {
+  if (!d) return PE_ERR_INVALID_ARG;
+  const int32_t V = d->num_ops, E = d->num_edges, D = d->num_devices, L = d->num_link_classes;
+  if (V < 1 || E < 0 || D < 1 || D > 255 || L < 1 || L > 254) return PE_ERR_INVALID_ARG;
+  if (!d->dur || (E > 0 && (!d->edge_src || !d->edge_dst))) return PE_ERR_INVALID_ARG;
+  if ((int64_t)E * L > (int64_t)INT32_MAX) return PE_ERR_INVALID_ARG;
+
+  int64_t tsum = 0, msum = 0;
+  for (int32_t i = 0; i < V; ++i) {
+    if (d->dur[i] < 0) return PE_ERR_RANGE;
+    tsum += d->dur[i];
+    if (d->mem_delta) msum += d->mem_delta[i] < 0 ? -(int64_t)d->mem_delta[i] : (int64_t)d->mem_delta[i];
+    if (d->mem_weight) {
+      if (d->mem_weight[i] < 0) return PE_ERR_RANGE;
+      msum += d->mem_weight[i];
+    }
+  }
+  std::vector<int32_t> indeg(V, 0), succ_ptr(V + 1, 0);
+  for (int32_t b = 0; b < E; ++b) {
+    const int32_t p = d->edge_src[b], i = d->edge_dst[b];
+    if (p < 0 || p >= V || i < 0 || i >= V) return PE_ERR_RANGE;
+    if (p == i) return PE_ERR_CYCLE;
+    indeg[i]++;
+    succ_ptr[p + 1]++;
+    if (d->comm) {
+      int32_t mx = 0;
+      for (int32_t l = 0; l < L; ++l) {
+        const int32_t cst = d->comm[(size_t)b * L + l];
+        if (cst < 0) return PE_ERR_RANGE;
+        if (cst > mx) mx = cst;
+      }
+      tsum += mx;
+    }
+  }
+  if (d->link_class)
+    for (int32_t a = 0; a < D * D; ++a)
+      if (d->link_class[a] != 0xFF && d->link_class[a] >= L) return PE_ERR_RANGE;
+  if (tsum > (int64_t)INT32_MAX || msum > (int64_t)INT32_MAX) return PE_ERR_OVERFLOW;
+
+  // acyclic iff Kahn's algorithm removes every operator
+  int32_t mdeg = 0;
+  for (int32_t i = 0; i < V; ++i) {
+    succ_ptr[i + 1] += succ_ptr[i];
+    if (indeg[i] > mdeg) mdeg = indeg[i];
+  }
+  std::vector<int32_t> succ(E), fill(succ_ptr.begin(), succ_ptr.end() - 1), deg(indeg), stack;
+  for (int32_t b = 0; b < E; ++b) succ[fill[d->edge_src[b]]++] = d->edge_dst[b];
+  for (int32_t i = 0; i < V; ++i)
+    if (deg[i] == 0) stack.push_back(i);
+  int32_t removed = 0;
+  while (!stack.empty()) {
+    const int32_t i = stack.back();
+    stack.pop_back();
+    ++removed;
+    for (int32_t q = succ_ptr[i]; q < succ_ptr[i + 1]; ++q)
+      if (--deg[succ[q]] == 0) stack.push_back(succ[q]);
+  }
+  if (removed != V) return PE_ERR_CYCLE;
+
+  if (time_bound) *time_bound = tsum;
+  if (mem_bound) *mem_bound = msum;
+  if (max_indeg) *max_indeg = mdeg;
+  return PE_OK;
+}
+
+}  // namespace
+
+extern "C" int pe_graph_validate(const pe_graph_desc* desc) { return check_desc(desc, nullptr, nullptr, nullptr); }
+
+extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph** out) {
+  if (!out) return PE_ERR_INVALID_ARG;
+  *out = nullptr;
+  int64_t tb = 0, mb = 0;
+  int32_t mdeg = 0;
+  const int rc = check_desc(d, &tb, &mb, &mdeg);
+  if (rc != PE_OK) return rc;
+  const int32_t V = d->num_ops, E = d->num_edges, D = d->num_devices, L = d->num_link_classes;
+
+  pe_graph* g = new (std::nothrow) pe_graph();
+  if (!g) return PE_ERR_INVALID_ARG;
+  g->V = V; g->E = E; g->D = D; g->L = L;
+  g->device = cuda_device;
+  g->has_weight = d->mem_weight != nullptr;
+  g->time_bound = tb; g->mem_bound = mb; g->max_indeg = mdeg;
+  g->d_blob = nullptr; g->d_error = nullptr;
+
+  PeBlobLayout& lay = g->lay;
+  uint64_t at = 0;
+  lay.ops = (uint32_t)at;    at = align16(at + (uint64_t)V * sizeof(PeOpRec));
+  lay.pred = (uint32_t)at;   at = align16(at + (uint64_t)E * 4);
+  lay.comm = (uint32_t)at;   at = align16(at + (uint64_t)E * L * 4);
+  lay.weight = (uint32_t)at; at = align16(at + (g->has_weight ? (uint64_t)V * 4 : 0));
+  lay.cls = (uint32_t)at;    at = align16(at + (uint64_t)D * D);
+  lay.cap = (uint32_t)at;    at = align16(at + (uint64_t)D * 4);
+  if (at > 0x7FFFFFF0ull) { delete g; return PE_ERR_INVALID_ARG; }
+  lay.bytes = (uint32_t)at;
+
+  // by-predecessor CSR: incoming edges of operator i occupy slots edge_begin .. edge_begin + indeg
+  std::vector<uint8_t> blob(lay.bytes, 0);
+  PeOpRec* ops = (PeOpRec*)(blob.data() + lay.ops);
+  int32_t* pred = (int32_t*)(blob.data() + lay.pred);
+  int32_t* comm = (int32_t*)(blob.data() + lay.comm);
+  for (int32_t i = 0; i < V; ++i) {
+    ops[i].indeg = 0;
+    ops[i].dur = d->dur[i];
+    ops[i].mem_delta = d->mem_delta ? d->mem_delta[i] : 0;
+  }
+  for (int32_t b = 0; b < E; ++b) ops[d->edge_dst[b]].indeg++;
+  int32_t run = 0;
+  for (int32_t i = 0; i < V; ++i) { ops[i].edge_begin = run; run += ops[i].indeg; }
+  {
+    std::vector<int32_t> fill(V);
+    for (int32_t i = 0; i < V; ++i) fill[i] = ops[i].edge_begin;
+    for (int32_t b = 0; b < E; ++b) {
+      const int32_t q = fill[d->edge_dst[b]]++;
+      pred[q] = d->edge_src[b];
+      for (int32_t l = 0; l < L; ++l) comm[(size_t)q * L + l] = d->comm ? d->comm[(size_t)b * L + l] : 0;
+    }
+  }
+  if (g->has_weight) std::memcpy(blob.data() + lay.weight, d->mem_weight, (size_t)V * 4);
+  if (d->link_class) std::memcpy(blob.data() + lay.cls, d->link_class, (size_t)D * D);
+  int32_t* cap = (int32_t*)(blob.data() + lay.cap);
+  for (int32_t j = 0; j < D; ++j) cap[j] = d->mem_capacity ? d->mem_capacity[j] : INT32_MAX;
+
+  cudaDeviceProp prop;
+  int prev = -1;
+  bool ok = cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(cuda_device) == cudaSuccess &&
+            cudaGetDeviceProperties(&prop, cuda_device) == cudaSuccess;
+  if (ok) {
+    g->sm_count = prop.multiProcessorCount;
+    g->smem_optin = prop.sharedMemPerBlockOptin;
+    ok = cudaMalloc((void**)&g->d_blob, lay.bytes) == cudaSuccess &&
+         cudaMalloc((void**)&g->d_error, 256) == cudaSuccess &&
+         cudaMemcpy(g->d_blob, blob.data(), lay.bytes, cudaMemcpyHostToDevice) == cudaSuccess &&
+         cudaMemset(g->d_error, 0, 256) == cudaSuccess;
+  }
+  if (prev >= 0) cudaSetDevice(prev);
+  if (!ok) {
+    cudaGetLastError();
+    if (g->d_blob) cudaFree(g->d_blob);
+    if (g->d_error) cudaFree(g->d_error);
+    delete g;
+    return PE_ERR_CUDA;
+  }
+  *out = g;
+  return PE_OK;
+}
+
+extern "C" int pe_destroy(pe_graph* g) {
+  if (!g) return PE_OK;
+  int prev = -1;
+  cudaGetDevice(&prev);
+  cudaSetDevice(g->device);
+  const bool ok = cudaFree(g->d_blob) == cudaSuccess && cudaFree(g->d_error) == cudaSuccess;
+  if (prev >= 0) cudaSetDevice(prev);
+  delete g;
+  return ok ? PE_OK : PE_ERR_CUDA;
+}
+
+extern "C" int pe_graph_poll_error(pe_graph* g, void* cuda_stream) {
+  if (!g) return PE_ERR_INVALID_ARG;
+  int word = 0;
+  if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return PE_ERR_CUDA;
+  if (cudaMemcpy(&word, g->d_error, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PE_ERR_CUDA;
+  if (word != 0 && cudaMemset(g->d_error, 0, sizeof(int)) != cudaSuccess) return PE_ERR_CUDA;
+  return word;
+}
+
+extern "C" const char* pe_strerror(int code) {
+  switch (code) {
+    case PE_OK: return "ok";
+    case PE_ERR_INVALID_ARG: return "invalid argument";
+    case PE_ERR_CYCLE: return "operator graph has a cycle";
+    case PE_ERR_RANGE: return "value out of range (negative duration/communication/weight, edge endpoint or link class)";
+    case PE_ERR_OVERFLOW: return "time or memory bound does not fit in int32";
+    case PE_ERR_CUDA: return "CUDA runtime call failed";
+    case PE_ERR_WORKSPACE: return "workspace missing or too small";
+    case PE_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case PE_ERR_UNSUPPORTED: return "kernel variant cannot run this problem size";
+    default: return "unknown error code";
+  }
+}

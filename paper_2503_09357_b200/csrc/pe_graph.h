@@ -1,0 +1,57 @@
+// Internal: host-side graph handle and the device-side view kernels receive.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "pe.h"
+
+// One record per operator i, 16 bytes: where its incoming edges start in the by-predecessor
+// CSR, how many there are, its duration D^o_i and its memory adjustment A_i.
+struct PeOpRec {
+  int32_t edge_begin;
+  int32_t indeg;
+  int32_t dur;
+  int32_t mem_delta;
+};
+
+// Byte offsets of the arrays inside the graph blob (one contiguous, 16-byte aligned block in
+// device memory, copied verbatim into shared memory by the kernels that stage it).
+struct PeBlobLayout {
+  uint32_t ops;     // PeOpRec[V]
+  uint32_t pred;    // int32[E]      predecessor id of CSR slot q
+  uint32_t comm;    // int32[E*L]    D^c of CSR slot q over link class l at q*L + l
+  uint32_t weight;  // int32[V]      W_i (present only if has_weight)
+  uint32_t cls;     // uint8[D*D]    link class of (machine of predecessor, machine of successor)
+  uint32_t cap;     // int32[D]      capacity (INT32_MAX where there is no limit)
+  uint32_t bytes;   // total, multiple of 16
+};
+
+// What a kernel needs to know about the graph; `base` points at the blob (global or shared).
+struct PeGraphView {
+  int32_t V, E, D, L;
+  int32_t has_weight;
+  PeBlobLayout lay;
+};
+
+struct pe_graph {
+  int32_t V, E, D, L;
+  int device;
+  bool has_weight;
+  int64_t time_bound;  // sum dur + sum_e max_l comm: no start/end time exceeds it
+  int64_t mem_bound;   // sum |A| + sum W
+  int32_t max_indeg;
+  PeBlobLayout lay;
+  uint8_t* d_blob;     // device copy of the blob
+  int* d_error;        // device status word (0 = ok)
+  int sm_count;
+  size_t smem_optin;   // max dynamic shared memory per block
+};
+
+inline PeGraphView pe_view(const pe_graph* g) {
+  PeGraphView v;
+  v.V = g->V; v.E = g->E; v.D = g->D; v.L = g->L;
+  v.has_weight = g->has_weight ? 1 : 0;
+  v.lay = g->lay;
+  return v;
+}

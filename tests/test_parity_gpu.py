@@ -1,0 +1,252 @@
+"""Parity of the CUDA path (through the C-ABI) with the CPU oracle: bit-exact on every output."""
+import numpy as np
+import pytest
+
+from paper_2503_09357_b200 import workloads as wl
+from tests import checkers as ck
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pe():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    from paper_2503_09357_b200 import binding
+    return binding
+
+
+def variants_for(pe, graph, K, base_flags=0):
+    out = [("auto", base_flags)]
+    for name, bit in (("global", pe.PE_VARIANT_GLOBAL), ("shared", pe.PE_VARIANT_SHARED), ("warp", pe.PE_VARIANT_WARP)):
+        if pe.pe_eval_variant(graph.handle, K, base_flags | bit) >= 0:
+            out.append((name, base_flags | bit))
+    return out
+
+
+# ---- the five configurations; 1-4 at full K, the sweep at K*V = 2^23 ----
+CASES = [(1, {}, None), (2, {}, None), (3, {}, None), (4, {}, None)] + \
+        [(5, dict(V=V, D=D), (1 << 23) // V) for V, D in wl.SWEEP_POINTS]
+
+
+@pytest.mark.parametrize("config,kw,K", CASES, ids=lambda v: str(v).replace(" ", ""))
+def test_configs_match_oracle(pe, config, kw, K):
+    w = wl.make_config(config, **kw)
+    K = w.num_candidates if K is None else K
+    assign, order = wl.make_candidates(w, K=K)
+    g = pe.Graph(w)
+    try:
+        seen = set()
+        for name, flags in variants_for(pe, g, K):
+            v = g.variant(K, flags)
+            if name == "auto":
+                seen.add(v)
+            elif v in seen and name != "auto" and K * w.num_ops > (1 << 24):
+                continue                                   # the auto run already covered this variant at full size
+            gpu, ref = gu.check(g, w, assign, order, flags=flags, label=f"config {config} {kw} {name}")
+            assert (ref["status"] & gu.INVALID == 0).all()
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("config,kw", [(1, {}), (3, {}), (5, dict(V=256, D=64)), (5, dict(V=1024, D=8))])
+@pytest.mark.parametrize("layout", ["assign_by_pos", "times_by_op", "both", "summary_only"])
+def test_layout_flags(pe, config, kw, layout):
+    w = wl.make_config(config, **kw)
+    K = 1000                                               # ragged: not a multiple of any block size
+    assign, order = wl.make_candidates(w, K=K)
+    g = pe.Graph(w)
+    try:
+        base = {"assign_by_pos": pe.PE_ASSIGN_BY_POS, "times_by_op": pe.PE_TIMES_BY_OP,
+                "both": pe.PE_ASSIGN_BY_POS | pe.PE_TIMES_BY_OP, "summary_only": 0}[layout]
+        a = wl.assign_by_pos(assign, order) if base & pe.PE_ASSIGN_BY_POS else assign
+        for name, flags in variants_for(pe, g, K, base):
+            gu.check(g, w, a, order, flags=flags, want_times=layout != "summary_only", label=f"{layout} {name}")
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("K", [0, 1, 31, 33, 257])
+def test_small_and_ragged_batches(pe, K):
+    w = wl.make_config(2)
+    g = pe.Graph(w)
+    try:
+        if K == 0:
+            o = pe.make_outputs()
+            assert pe.pe_eval_batch(g.handle, 0, 0, 0, 2, 0, o) == pe.PE_OK
+            return
+        assign, order = wl.make_candidates(w, K=K)
+        for name, flags in variants_for(pe, g, K):
+            gu.check(g, w, assign, order, flags=flags, label=f"K={K} {name}")
+    finally:
+        g.close()
+
+
+def test_degenerate_graphs(pe):
+    cases = [
+        ck.problem(1, [], [5], 1, A=[2], cap=[1]),                                  # one op, one machine, over capacity
+        ck.problem(6, [], [1, 2, 3, 4, 5, 6], 3, A=[1, 1, 1, -1, -1, -1]),          # no edges
+        ck.problem(5, [(0, 4), (1, 4), (2, 4), (3, 4), (0, 4)], [1, 0, 2, 0, 3], 2, comm=2),   # duplicate edge, zero durations
+        ck.problem(4, [(0, 1), (1, 2), (2, 3)], [1, 1, 1, 1], 255, comm=3),         # D = 255
+    ]
+    for n, w in enumerate(cases):
+        w.assign_mode, w.group = "per_op", None
+        K = 77
+        assign, order = wl.make_candidates(w, K=K)
+        g = pe.Graph(w)
+        try:
+            for name, flags in variants_for(pe, g, K):
+                gu.check(g, w, assign, order, flags=flags, label=f"degenerate {n} {name}")
+        finally:
+            g.close()
+
+
+def test_weights_link_classes_and_missing_channels(pe):
+    w = wl.make_config(3)
+    w.mem_weight = (np.arange(w.num_ops) % 7).astype(np.int32)
+    w.link_class = w.link_class.copy()
+    w.link_class[3, 12] = 0xFF                              # one directed pair without a channel
+    w.mem_capacity = np.full(w.num_devices, 760, np.int32)   # near the typical per-machine peak: both outcomes occur
+    K = 512
+    assign, order = wl.make_candidates(w, K=K)
+    g = pe.Graph(w)
+    try:
+        for name, flags in variants_for(pe, g, K):
+            gpu, ref = gu.check(g, w, assign, order, flags=flags, label=f"weights {name}")
+            assert (ref["status"] & pe.PE_STATUS_NO_CHANNEL).any()
+            exceeded = (ref["status"] & pe.PE_STATUS_MEM_EXCEEDED) != 0
+            assert exceeded.any() and not exceeded.all()
+    finally:
+        g.close()
+
+
+def test_u32_orders(pe):
+    w = wl.make_config(5, V=1024, D=8)
+    K = 300
+    assign, order = wl.make_candidates(w, K=K, order_bytes=4)
+    assert order.dtype == np.uint32
+    g = pe.Graph(w)
+    try:
+        for name, flags in variants_for(pe, g, K):
+            gu.check(g, w, assign, order, flags=flags, label=f"u32 {name}")
+    finally:
+        g.close()
+
+
+def test_invalid_candidates_are_flagged_and_stay_in_bounds(pe):
+    w = wl.make_config(1)
+    K = 64
+    assign, order = wl.make_candidates(w, K=K)
+    assign, order = assign.copy(), order.copy()
+    order[[3, 40], 1] = order[[40, 3], 1]          # may or may not break a dependency; the oracle decides
+    order[5, 2] = order[4, 2]                      # duplicate (and so a missing op)
+    order[7, 3] = 60000                            # id out of range
+    assign[:, 4] = 200                             # machine id out of range
+    assign[9, 5] = 4                               # one machine id = D
+    order[:, 6] = order[::-1, 6].copy()            # reversed: every dependency broken
+    g = pe.Graph(w)
+    try:
+        for base in (0, pe.PE_ASSIGN_BY_POS):
+            a = wl.assign_by_pos(assign, order) if base else assign
+            for name, flags in variants_for(pe, g, K, base):
+                gpu, ref = gu.check(g, w, a, order, flags=flags, label=f"invalid {name}")
+                assert (ref["status"][[2, 3, 6]] & pe.PE_STATUS_ORDER_INVALID).all()
+                assert (ref["status"][[4, 5]] & pe.PE_STATUS_ASSIGN_RANGE).all()
+                assert (ref["status"][8:] == gpu["status"][8:]).all()
+    finally:
+        g.close()
+
+
+def test_large_time_bound_falls_back_to_the_global_variant(pe):
+    w = wl.make_config(5, V=256, D=8)
+    w.dur = (w.dur.astype(np.int64) * 100000).astype(np.int32)       # sum of durations ~ 1.3e9 < 2^31
+    K = 200
+    assign, order = wl.make_candidates(w, K=K)
+    g = pe.Graph(w)
+    try:
+        assert g.variant(K) == "global"
+        assert pe.pe_eval_variant(g.handle, K, pe.PE_VARIANT_SHARED) == pe.PE_ERR_UNSUPPORTED
+        gu.check(g, w, assign, order, label="large times")
+    finally:
+        g.close()
+
+
+def test_workspace_is_checked(pe):
+    import torch
+    w = wl.make_config(1)
+    K = 128
+    assign, order = wl.make_candidates(w, K=K)
+    g = pe.Graph(w)
+    try:
+        flags = pe.PE_VARIANT_GLOBAL
+        need = pe.pe_workspace_bytes(g.handle, K, flags)
+        assert need >= w.num_ops * K * 4
+        a = torch.from_numpy(assign).cuda(); o = torch.from_numpy(gu.as_signed(order)).cuda()
+        out = g.alloc_outputs(K)
+        outs = pe.make_outputs(**{k: v.data_ptr() for k, v in out.items()})
+        ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        assert pe.pe_eval_batch(g.handle, K, a.data_ptr(), o.data_ptr(), 2, flags, outs, ws.data_ptr(), need - 1, 0) == pe.PE_ERR_WORKSPACE
+        assert pe.pe_eval_batch(g.handle, K, a.data_ptr(), o.data_ptr(), 2, flags, outs, 0, 0, 0) == pe.PE_ERR_WORKSPACE
+        assert pe.pe_eval_batch(g.handle, K, a.data_ptr(), o.data_ptr(), 3, flags, outs, ws.data_ptr(), need, 0) == pe.PE_ERR_INVALID_ARG
+        assert pe.pe_eval_batch(g.handle, K, a.data_ptr(), o.data_ptr(), 2, 1 << 20, outs, ws.data_ptr(), need, 0) == pe.PE_ERR_INVALID_ARG
+        assert pe.pe_graph_poll_error(g.handle, 0) == pe.PE_OK
+    finally:
+        g.close()
+
+
+def test_host_buffer_entry_point(pe):
+    import torch
+    w = wl.make_config(2)
+    K = 4096
+    V, D = w.num_ops, w.num_devices
+    assign, order = wl.make_candidates(w, K=K)
+    g = pe.Graph(w)
+    try:
+        h_a = torch.from_numpy(assign).pin_memory(); h_o = torch.from_numpy(gu.as_signed(order)).pin_memory()
+        d_a = torch.empty_like(h_a, device="cuda"); d_o = torch.empty_like(h_o, device="cuda")
+        d_out = g.alloc_outputs(K)
+        h_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in d_out.items()}
+        ws, ws_bytes = g.alloc_workspace(K)
+        before = pe.pe_kernel_launches()
+        rc = pe.pe_eval_batch_host(g.handle, K, h_a.data_ptr(), h_o.data_ptr(), 2, 0,
+                                   pe.make_outputs(**{k: v.data_ptr() for k, v in h_out.items()}),
+                                   d_a.data_ptr(), d_o.data_ptr(),
+                                   pe.make_outputs(**{k: v.data_ptr() for k, v in d_out.items()}),
+                                   ws.data_ptr(), ws_bytes, torch.cuda.current_stream().cuda_stream)
+        assert rc == pe.PE_OK and pe.pe_kernel_launches() == before + 1
+        res = {k: v.numpy() for k, v in h_out.items()}
+        res["status"] = res["status"].view(np.uint32)
+        from oracle import pe_oracle as orc
+        gu.compare(res, orc.evaluate(w, assign, order, threads=gu.CPU_THREADS), "host entry point")
+    finally:
+        g.close()
+
+
+def test_bench_configuration_sampled(pe):
+    """The benchmark's own launch (sweep point V=16384, D=64 at its full K) on sampled candidates:
+    every output of 512 randomly chosen candidates against the oracle, plus size-independent
+    properties on all of them."""
+    import torch
+    w = wl.make_config(5, V=16384, D=64)
+    K = w.num_candidates
+    assign, order = wl.make_candidates(w, K=K)
+    g = pe.Graph(w)
+    try:
+        gpu = gu.gpu_eval(g, assign, order)
+        rs = np.random.RandomState(5)
+        sample = np.sort(rs.choice(K, 512, replace=False))
+        from oracle import pe_oracle as orc
+        ref = orc.evaluate(w, np.ascontiguousarray(assign[:, sample]), np.ascontiguousarray(order[:, sample]),
+                           threads=gu.CPU_THREADS)
+        sub = {k: (v[sample] if v.ndim == 1 else v[:, sample]) for k, v in gpu.items()}
+        gu.compare(sub, ref, "bench configuration sample")
+        total = int(w.dur.astype(np.int64).sum())
+        assert (gpu["status"] == 0).all()
+        assert (gpu["busy"].sum(axis=0) == total).all()
+        assert np.array_equal(gpu["makespan"], gpu["finish"].max(axis=0))
+        assert (gpu["finish"] - gpu["start"] == w.dur[order.astype(np.int64)]).all()
+        assert (gpu["makespan"] >= gpu["busy"].max(axis=0)).all() and (gpu["makespan"] >= ck.critical_path(w)).all()
+    finally:
+        g.close()
