@@ -46,7 +46,8 @@ enum {
   PE_ERR_CUDA = -5,        /* a CUDA runtime call failed (no device, out of memory, launch error) */
   PE_ERR_WORKSPACE = -6,   /* workspace pointer NULL or smaller than pe_workspace_bytes() */
   PE_ERR_TIMEOUT = -7,     /* a bounded device-side wait expired (reported by pe_graph_poll_error) */
-  PE_ERR_UNSUPPORTED = -8  /* the requested kernel variant cannot run this problem size */
+  PE_ERR_UNSUPPORTED = -8, /* the requested kernel variant cannot run this problem size */
+  PE_ERR_SCRATCH_LIMIT = -9 /* pe_eval_batch_noalloc: the batch needs more than PE_NOALLOC_SCRATCH_BYTES of scratch */
 };
 
 /* Problem data (Section III).  All pointers are HOST pointers, read during the call only. */
@@ -133,6 +134,37 @@ int pe_eval_batch(pe_graph* g, int64_t K, const uint8_t* assign, const void* ord
 int pe_eval_batch_host(pe_graph* g, int64_t K, const uint8_t* host_assign, const void* host_order, int order_bytes,
                        uint32_t flags, const pe_outputs* host_out, uint8_t* dev_assign, void* dev_order,
                        const pe_outputs* dev_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Evaluation for callers that must not allocate device memory.  (The paper has no counterpart:
+ * this is a convenience of the library, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a memory pool or framework
+ * that owns every byte of the device and forbids side allocations, in a latency-critical loop
+ * where an allocation would synchronise the device, or in a process whose memory budget was fixed
+ * at start-up.  pe_eval_batch asks such a caller for a workspace it cannot provide; this entry
+ * point brings its own.
+ *
+ * It runs the one-thread-per-candidate kernel whose per-operator state lives in global memory
+ * (the PE_VARIANT_GLOBAL kernel), with that state in a fixed array of PE_NOALLOC_SCRATCH_BYTES
+ * that is part of the library image: every GPU on which the library is used holds it from the
+ * first use until the process exits.  Inputs and outputs are still the caller's device buffers,
+ * with the meaning and layouts of pe_eval_batch; flags may hold PE_ASSIGN_BY_POS and
+ * PE_TIMES_BY_OP only (no variant bits).  Results are identical to pe_eval_batch's.
+ *
+ *  - Size limit: pe_workspace_bytes(g, K, flags | PE_VARIANT_GLOBAL) must not exceed
+ *    PE_NOALLOC_SCRATCH_BYTES (about 4*V*K bytes, 5*V*K with PE_ASSIGN_BY_POS); a larger batch is
+ *    refused with PE_ERR_SCRATCH_LIMIT and nothing is launched.  Split the batch instead.
+ *  - The first call on each device looks up the array's device address (a short, synchronous
+ *    set-up with that device current); make that first call before starting any stream capture.
+ *  - No cudaMalloc, cudaFree or other allocating routine is called, on any call.
+ *  - All calls share the one array per device.  Each call re-initialises the part it uses on
+ *    `cuda_stream` before its kernel, so stale contents never leak into a result; but two calls
+ *    that can overlap on the GPU (different streams, or different host threads without ordering)
+ *    race on it and give wrong results.  Order them on one stream or with events.
+ * Asynchronous on `cuda_stream`, like pe_eval_batch. */
+#define PE_NOALLOC_SCRATCH_BYTES (64u << 20)
+int pe_eval_batch_noalloc(pe_graph* g, int64_t K, const uint8_t* assign, const void* order, int order_bytes,
+                          uint32_t flags, const pe_outputs* out, void* cuda_stream);
 
 /* Synchronise `cuda_stream` and return the graph's device-side error word: PE_OK, or
  * PE_ERR_TIMEOUT if a kernel gave up a bounded wait (its outputs are then invalid).  Clears the word. */

@@ -22,6 +22,8 @@ _lib = ctypes.CDLL(LIB_PATH)
 PE_OK = 0
 PE_ERR_INVALID_ARG, PE_ERR_CYCLE, PE_ERR_RANGE, PE_ERR_OVERFLOW = -1, -2, -3, -4
 PE_ERR_CUDA, PE_ERR_WORKSPACE, PE_ERR_TIMEOUT, PE_ERR_UNSUPPORTED = -5, -6, -7, -8
+PE_ERR_SCRATCH_LIMIT = -9
+PE_NOALLOC_SCRATCH_BYTES = 64 << 20
 PE_ASSIGN_BY_POS, PE_TIMES_BY_OP = 1, 2
 PE_VARIANT_AUTO, PE_VARIANT_GLOBAL, PE_VARIANT_SHARED, PE_VARIANT_WARP = 0 << 8, 1 << 8, 2 << 8, 3 << 8
 PE_VARIANT_MASK = 15 << 8
@@ -58,6 +60,9 @@ _lib.pe_eval_batch_host.restype = ctypes.c_int
 _lib.pe_eval_batch_host.argtypes = [_P, ctypes.c_int64, _P, _P, ctypes.c_int, ctypes.c_uint32,
                                     ctypes.POINTER(pe_outputs), _P, _P, ctypes.POINTER(pe_outputs), _P,
                                     ctypes.c_size_t, _P]
+_lib.pe_eval_batch_noalloc.restype = ctypes.c_int
+_lib.pe_eval_batch_noalloc.argtypes = [_P, ctypes.c_int64, _P, _P, ctypes.c_int, ctypes.c_uint32,
+                                       ctypes.POINTER(pe_outputs), _P]
 _lib.pe_graph_poll_error.restype = ctypes.c_int
 _lib.pe_graph_poll_error.argtypes = [_P, _P]
 _lib.pe_kernel_launches.restype = ctypes.c_int64
@@ -153,6 +158,13 @@ def pe_eval_batch_host(handle, K, host_assign_ptr, host_order_ptr, order_bytes, 
     return _lib.pe_eval_batch_host(handle, int(K), host_assign_ptr, host_order_ptr, int(order_bytes), int(flags),
                                    ctypes.byref(host_outputs), dev_assign_ptr, dev_order_ptr, ctypes.byref(dev_outputs),
                                    workspace_ptr or None, int(workspace_bytes), stream or None)
+
+
+def pe_eval_batch_noalloc(handle, K, assign_ptr, order_ptr, order_bytes, flags, outputs, stream=0) -> int:
+    """Raw call of the entry point that brings its own scratch (for callers that cannot allocate
+    device memory); same pointer conventions as pe_eval_batch, no workspace argument."""
+    return _lib.pe_eval_batch_noalloc(handle, int(K), assign_ptr or None, order_ptr or None, int(order_bytes),
+                                      int(flags), ctypes.byref(outputs), stream or None)
 
 
 def pe_graph_poll_error(handle, stream=0) -> int:

@@ -382,3 +382,67 @@ extern "C" int pe_eval_batch_host(pe_graph* g, int64_t K, const uint8_t* host_as
   if (prev != g->device) cudaSetDevice(prev);
   return ret;
 }
+
+// ============================================================================================
+// pe_eval_batch_noalloc: the GLOBAL variant with its scratch in an array that is part of the
+// library image, for callers that may not allocate device memory.
+// ============================================================================================
+namespace pe {
+
+// The scratch itself.  In host code this name is only a handle for the runtime's symbol
+// lookup, never a device address: the address kernels and memsets need comes from
+// cudaGetSymbolAddress, looked up once per device below.
+static __device__ __align__(256) uint8_t g_noalloc_scratch[PE_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+static std::atomic<void*> g_noalloc_addr[kMaxDevices];
+
+// Device address of the scratch array on `device`, which must be the current device.
+static int noalloc_scratch_address(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return PE_ERR_INVALID_ARG;
+  void* p = g_noalloc_addr[device].load(std::memory_order_acquire);
+  if (!p) {
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return PE_ERR_CUDA;
+    }
+    g_noalloc_addr[device].store(p, std::memory_order_release);  // every thread resolves the same address
+  }
+  *out = p;
+  return PE_OK;
+}
+
+}  // namespace pe
+
+extern "C" int pe_eval_batch_noalloc(pe_graph* g, int64_t K, const uint8_t* assign, const void* order, int order_bytes,
+                                     uint32_t flags, const pe_outputs* out, void* cuda_stream) {
+  if (!g || !out || K < 0) return PE_ERR_INVALID_ARG;
+  if (order_bytes != 2 && order_bytes != 4) return PE_ERR_INVALID_ARG;
+  if (order_bytes == 2 && g->V > 65536) return PE_ERR_INVALID_ARG;
+  if (flags & ~(uint32_t)(PE_ASSIGN_BY_POS | PE_TIMES_BY_OP)) return PE_ERR_INVALID_ARG;
+  pe::Plan p;
+  if (!pe::plan_global(g, K, flags, &p)) return PE_ERR_UNSUPPORTED;
+  if (p.workspace > (size_t)PE_NOALLOC_SCRATCH_BYTES) return PE_ERR_SCRATCH_LIMIT;
+  if (K == 0) return PE_OK;
+  if (!assign || !order) return PE_ERR_INVALID_ARG;
+  if ((K + p.threads - 1) / p.threads > (int64_t)INT_MAX) return PE_ERR_INVALID_ARG;
+  int prev = -1;
+  if (cudaGetDevice(&prev) != cudaSuccess) return PE_ERR_CUDA;
+  if (prev != g->device && cudaSetDevice(g->device) != cudaSuccess) return PE_ERR_CUDA;
+  void* scratch = nullptr;
+  int ret = pe::noalloc_scratch_address(g->device, &scratch);
+  if (ret == PE_OK) {
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const bool by_pos = (flags & PE_ASSIGN_BY_POS) != 0;
+    // launch_typed clears the end-time state (the part of the scratch that must start as "not
+    // scheduled") on the stream before the kernel, so the previous call's contents never matter
+    if (order_bytes == 2)
+      ret = by_pos ? pe::launch_typed<uint16_t, true>(g, p, K, assign, order, flags, *out, scratch, stream)
+                   : pe::launch_typed<uint16_t, false>(g, p, K, assign, order, flags, *out, scratch, stream);
+    else
+      ret = by_pos ? pe::launch_typed<uint32_t, true>(g, p, K, assign, order, flags, *out, scratch, stream)
+                   : pe::launch_typed<uint32_t, false>(g, p, K, assign, order, flags, *out, scratch, stream);
+  }
+  if (prev != g->device) cudaSetDevice(prev);
+  return ret;
+}

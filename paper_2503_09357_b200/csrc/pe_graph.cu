@@ -191,6 +191,7 @@ extern "C" const char* pe_strerror(int code) {
     case PE_ERR_WORKSPACE: return "workspace missing or too small";
     case PE_ERR_TIMEOUT: return "bounded device-side wait expired";
     case PE_ERR_UNSUPPORTED: return "kernel variant cannot run this problem size";
+    case PE_ERR_SCRATCH_LIMIT: return "batch needs more scratch than the built-in no-allocation array holds";
     default: return "unknown error code";
   }
 }

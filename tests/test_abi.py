@@ -74,7 +74,7 @@ def test_validate_codes(pe):
 
 
 def test_strerror_and_null_handles(pe):
-    for code in range(-8, 1):
+    for code in range(-9, 1):
         assert "unknown" not in pe.pe_strerror(code)
     assert "unknown" in pe.pe_strerror(-99)
     assert pe.pe_destroy(None) == pe.PE_OK
