@@ -187,7 +187,8 @@ def run_ours(args):
     w = WORKLOADS[args.workload]()
     V, D, K = w.num_ops, w.num_devices, (args.candidates or w.num_candidates)
     want_times = args.outputs == "full"
-    flags = 0
+    flags = {"auto": pe.PE_VARIANT_AUTO, "global": pe.PE_VARIANT_GLOBAL, "shared": pe.PE_VARIANT_SHARED,
+             "warp": pe.PE_VARIANT_WARP}[args.variant]
     obytes = 2 if V <= 65536 else 4
     odt = torch.int16 if obytes == 2 else torch.int32
 
@@ -329,6 +330,8 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default=DEFAULT_WORKLOAD)
     ap.add_argument("--outputs", choices=["full", "summary"], default="full")
+    ap.add_argument("--variant", choices=["auto", "global", "shared", "warp"], default="auto",
+                    help="force a kernel variant (default: the library chooses)")
     ap.add_argument("--candidates", type=int, default=0, help="override K per GPU (default: the configuration's K)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)

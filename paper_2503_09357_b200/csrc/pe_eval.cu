@@ -12,6 +12,8 @@
 
 #include "pe_device.cuh"
 #include "pe_graph.h"
+#include "pe_kernel_lane.cuh"
+#include "pe_kernel_warp.cuh"
 
 namespace pe {
 
@@ -200,18 +202,37 @@ __global__ void pe_eval_shared_kernel(PeGraphView g, const uint8_t* __restrict__
 // Host-side planning: which variant, with what launch shape.
 // ============================================================================================
 struct Plan {
-  int variant;        // PE_VARIANT_* value
-  int threads;        // block size
-  size_t smem;        // dynamic shared memory per block
-  bool graph_smem;    // graph blob staged into shared memory
-  size_t workspace;   // bytes of caller workspace
-  size_t ws_x_off;    // offset of the machine-state array inside the workspace (GLOBAL, by-pos)
+  int variant = 0;        // PE_VARIANT_* value
+  int threads = 0;        // block size
+  size_t smem = 0;        // dynamic shared memory per block
+  bool graph_smem = false;  // graph blob staged into shared memory
+  size_t workspace = 0;   // bytes of caller workspace
+  size_t ws_x_off = 0;    // offset of the machine-state array inside the workspace (generic GLOBAL, by-pos)
+  int warp_words = 0;     // WARP: 32-bit words of shared memory per candidate
+  bool compact = false;   // SHARED / GLOBAL: the compact-graph kernel (pe_eval_lane_kernel)
 };
 
 static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-static bool plan_shared(const pe_graph* g, Plan* p) {
+static bool plan_shared(const pe_graph* g, bool allow_compact, Plan* p) {
   if (g->time_bound >= kPackedTimeLimit) return false;
+  p->compact = false;
+  if (g->narrow_ok && allow_compact) {  // compact graph staged in shared memory next to the state
+    const size_t per = (size_t)4 * (g->V + 1) + (size_t)(g->has_weight ? 20 : 16) * g->D;
+    const size_t fixed = (size_t)g->nview.bytes + 16;
+    if (fixed + 32 * per <= g->smem_optin) {
+      size_t T = (g->smem_optin - fixed) / per / 32 * 32;
+      if (T > 256) T = 256;
+      p->variant = PE_VARIANT_SHARED;
+      p->threads = (int)T;
+      p->smem = fixed + T * per;
+      p->graph_smem = true;
+      p->workspace = 0;
+      p->ws_x_off = 0;
+      p->compact = true;
+      return true;
+    }
+  }
   const size_t per_thread = (size_t)4 * g->V + (size_t)(g->has_weight ? 20 : 16) * g->D;
   const size_t budget = g->smem_optin;
   for (int with_graph = 1; with_graph >= 0; --with_graph) {
@@ -230,7 +251,51 @@ static bool plan_shared(const pe_graph* g, Plan* p) {
   return false;
 }
 
-static bool plan_global(const pe_graph* g, int64_t K, uint32_t flags, Plan* p) {
+static bool plan_warp(const pe_graph* g, Plan* p) {
+  if (g->time_bound >= kPackedTimeLimit) return false;
+  p->compact = false;
+  size_t words = (size_t)(g->V | 1) + (size_t)5 * g->D;
+  words |= 1;  // odd stride between candidates: the initial fill hits distinct banks
+  const size_t per_warp = words * 4;
+  const size_t budget = g->smem_optin;
+  auto fit = [&](size_t fixed) -> int {
+    if (fixed + per_warp > budget) return 0;
+    const size_t n = (budget - fixed) / per_warp;
+    return (int)(n > 32 ? 32 : n);
+  };
+  const int n_global = fit(0);
+  const int n_staged = fit((size_t)g->lay.bytes + 16);
+  if (n_global < 1) return false;
+  const bool staged = n_staged >= (n_global < 8 ? n_global : 8);
+  const int n = staged ? n_staged : n_global;
+  p->variant = PE_VARIANT_WARP;
+  p->threads = 32 * n;
+  p->smem = (staged ? (size_t)g->lay.bytes + 16 : 0) + (size_t)n * per_warp;
+  p->graph_smem = staged;
+  p->workspace = 0;
+  p->ws_x_off = 0;
+  p->warp_words = (int)words;
+  return true;
+}
+
+static bool plan_global(const pe_graph* g, int64_t K, uint32_t flags, bool allow_compact, Plan* p) {
+  p->compact = false;
+  if (g->narrow_ok && allow_compact && g->time_bound < kPackedTimeLimit) {
+    // compact-graph kernel with the state in the workspace; small blocks so that several fit on an SM
+    const size_t per = (size_t)(g->has_weight ? 20 : 16) * g->D;
+    size_t T = 128;
+    while (T > 32 && T * per > 32768) T /= 2;
+    if (T * per <= g->smem_optin) {
+      p->variant = PE_VARIANT_GLOBAL;
+      p->threads = (int)T;
+      p->smem = T * per;
+      p->graph_smem = false;
+      p->ws_x_off = 0;
+      p->workspace = round_up((size_t)(g->V + 1) * (size_t)K * 4, 256);
+      p->compact = true;
+      return true;
+    }
+  }
   const size_t per_thread = (size_t)20 * g->D;
   size_t T = g->smem_optin / per_thread / 32 * 32;
   if (T > 128) T = 128;
@@ -244,16 +309,23 @@ static bool plan_global(const pe_graph* g, int64_t K, uint32_t flags, Plan* p) {
   return true;
 }
 
-static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, Plan* p) {
+// allow_compact: the call can use the compact-graph kernels (u16 orders; start and finish both
+// wanted or both absent).  Size queries pass true and false and take the larger workspace.
+static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, bool allow_compact, Plan* p) {
   if (!g || K < 0) return PE_ERR_INVALID_ARG;
   if (flags & ~(uint32_t)(PE_ASSIGN_BY_POS | PE_TIMES_BY_OP | PE_VARIANT_MASK)) return PE_ERR_INVALID_ARG;
+  *p = Plan();
   const uint32_t want = flags & PE_VARIANT_MASK;
   switch (want) {
     case PE_VARIANT_AUTO:
-      if (plan_shared(g, p)) return PE_OK;
-      return plan_global(g, K, flags, p) ? PE_OK : PE_ERR_UNSUPPORTED;
-    case PE_VARIANT_GLOBAL: return plan_global(g, K, flags, p) ? PE_OK : PE_ERR_UNSUPPORTED;
-    case PE_VARIANT_SHARED: return plan_shared(g, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+      if (plan_shared(g, allow_compact, p) && p->threads >= 64) return PE_OK;
+      if (plan_global(g, K, flags, allow_compact, p) && p->compact) return PE_OK;
+      if (plan_warp(g, p)) return PE_OK;
+      if (plan_shared(g, allow_compact, p)) return PE_OK;
+      return plan_global(g, K, flags, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+    case PE_VARIANT_GLOBAL: return plan_global(g, K, flags, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+    case PE_VARIANT_SHARED: return plan_shared(g, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+    case PE_VARIANT_WARP: return plan_warp(g, p) ? PE_OK : PE_ERR_UNSUPPORTED;
     default: return PE_ERR_UNSUPPORTED;
   }
 }
@@ -263,13 +335,57 @@ static bool set_smem(Kern kern, size_t bytes) {
   return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
 }
 
+// The compact-graph kernel: state in shared memory (SHARED) or in the workspace (GLOBAL).
+template <typename IdxT, bool BY_POS, int CLS, bool STATE_SMEM>
+static int launch_compact4(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* assign, const uint16_t* order,
+                           uint32_t flags, const pe_outputs& out, uint32_t* gstate, unsigned grid,
+                           cudaStream_t stream) {
+  auto go = [&](auto kern) -> int {
+    if (!set_smem(kern, p.smem)) return PE_ERR_CUDA;
+    kern<<<grid, p.threads, p.smem, stream>>>(g->nview, g->d_nblob, K, assign, order, out, flags, g->d_error, gstate);
+    return PE_OK;
+  };
+  return out.start ? go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, true>)
+                   : go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, false>);
+}
+
+template <bool BY_POS>
+static int launch_compact(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* assign, const uint16_t* order,
+                          uint32_t flags, const pe_outputs& out, uint32_t* gstate, unsigned grid,
+                          cudaStream_t stream) {
+  const bool smem_state = p.variant == PE_VARIANT_SHARED;
+  const bool idx32 = (uint64_t)(g->V + 1) * (uint64_t)K <= 0xFFFFFFFFull;
+  const int cls = g->nview.L == 2 ? 2 : (g->nview.need_cls ? 1 : 0);
+#define PE_GO(IDX, CLS, SM) return launch_compact4<IDX, BY_POS, CLS, SM>(g, p, K, assign, order, flags, out, gstate, grid, stream)
+#define PE_GO_CLS(IDX, SM)        \
+  do {                            \
+    if (cls == 2) PE_GO(IDX, 2, SM); \
+    if (cls == 1) PE_GO(IDX, 1, SM); \
+    PE_GO(IDX, 0, SM);            \
+  } while (0)
+  if (idx32) {
+    if (smem_state) PE_GO_CLS(uint32_t, true);
+    PE_GO_CLS(uint32_t, false);
+  }
+  if (smem_state) PE_GO_CLS(uint64_t, true);
+  PE_GO_CLS(uint64_t, false);
+#undef PE_GO_CLS
+#undef PE_GO
+}
+
 template <typename OrderT, bool BY_POS>
 static int launch_typed(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* assign, const void* order,
                         uint32_t flags, const pe_outputs& out, void* workspace, cudaStream_t stream) {
   const PeGraphView view = pe_view(g);
-  const unsigned grid = (unsigned)((K + p.threads - 1) / p.threads);
+  const int per_block = p.variant == PE_VARIANT_WARP ? p.threads / 32 : p.threads;  // candidates per block
+  const unsigned grid = (unsigned)((K + per_block - 1) / per_block);
   const OrderT* ord = static_cast<const OrderT*>(order);
-  if (p.variant == PE_VARIANT_GLOBAL) {
+  if (p.compact) {
+    if (sizeof(OrderT) != 2) return PE_ERR_INVALID_ARG;
+    const int rc = launch_compact<BY_POS>(g, p, K, assign, static_cast<const uint16_t*>(order), flags, out,
+                                          static_cast<uint32_t*>(workspace), grid, stream);
+    if (rc != PE_OK) return rc;
+  } else if (p.variant == PE_VARIANT_GLOBAL) {
     int32_t* e_state = static_cast<int32_t*>(workspace);
     uint8_t* x_state = static_cast<uint8_t*>(workspace) + p.ws_x_off;
     if (cudaMemsetAsync(e_state, 0xFF, (size_t)g->V * (size_t)K * 4, stream) != cudaSuccess) return PE_ERR_CUDA;
@@ -286,6 +402,16 @@ static int launch_typed(const pe_graph* g, const Plan& p, int64_t K, const uint8
       if (!set_smem(kern, p.smem)) return PE_ERR_CUDA;
       kern<<<grid, p.threads, p.smem, stream>>>(view, g->d_blob, K, assign, ord, out, flags, g->d_error);
     }
+  } else if (p.variant == PE_VARIANT_WARP) {
+    if (p.graph_smem) {
+      auto kern = pe_eval_warp_kernel<OrderT, BY_POS, true>;
+      if (!set_smem(kern, p.smem)) return PE_ERR_CUDA;
+      kern<<<grid, p.threads, p.smem, stream>>>(view, g->d_blob, K, assign, ord, out, flags, g->d_error, p.warp_words);
+    } else {
+      auto kern = pe_eval_warp_kernel<OrderT, BY_POS, false>;
+      if (!set_smem(kern, p.smem)) return PE_ERR_CUDA;
+      kern<<<grid, p.threads, p.smem, stream>>>(view, g->d_blob, K, assign, ord, out, flags, g->d_error, p.warp_words);
+    }
   } else {
     return PE_ERR_UNSUPPORTED;
   }
@@ -296,14 +422,15 @@ static int launch_typed(const pe_graph* g, const Plan& p, int64_t K, const uint8
 }  // namespace pe
 
 extern "C" size_t pe_workspace_bytes(const pe_graph* g, int64_t K, uint32_t flags) {
-  pe::Plan p;
-  if (pe::make_plan(g, K, flags, &p) != PE_OK) return 0;
-  return p.workspace;
+  pe::Plan a, b;
+  const size_t wa = pe::make_plan(g, K, flags, true, &a) == PE_OK ? a.workspace : 0;
+  const size_t wb = pe::make_plan(g, K, flags, false, &b) == PE_OK ? b.workspace : 0;
+  return wa > wb ? wa : wb;
 }
 
 extern "C" int pe_eval_variant(const pe_graph* g, int64_t K, uint32_t flags) {
   pe::Plan p;
-  const int rc = pe::make_plan(g, K, flags, &p);
+  const int rc = pe::make_plan(g, K, flags, true, &p);
   return rc != PE_OK ? rc : p.variant;
 }
 
@@ -316,7 +443,8 @@ extern "C" int pe_eval_batch(pe_graph* g, int64_t K, const uint8_t* assign, cons
   if (order_bytes != 2 && order_bytes != 4) return PE_ERR_INVALID_ARG;
   if (order_bytes == 2 && g->V > 65536) return PE_ERR_INVALID_ARG;
   pe::Plan p;
-  const int rc = pe::make_plan(g, K, flags, &p);
+  const bool allow_compact = order_bytes == 2 && ((out->start != nullptr) == (out->finish != nullptr));
+  const int rc = pe::make_plan(g, K, flags, allow_compact, &p);
   if (rc != PE_OK) return rc;
   if (K == 0) return PE_OK;
   if (!assign || !order) return PE_ERR_INVALID_ARG;
@@ -421,7 +549,8 @@ extern "C" int pe_eval_batch_noalloc(pe_graph* g, int64_t K, const uint8_t* assi
   if (order_bytes == 2 && g->V > 65536) return PE_ERR_INVALID_ARG;
   if (flags & ~(uint32_t)(PE_ASSIGN_BY_POS | PE_TIMES_BY_OP)) return PE_ERR_INVALID_ARG;
   pe::Plan p;
-  if (!pe::plan_global(g, K, flags, &p)) return PE_ERR_UNSUPPORTED;
+  const bool allow_compact = order_bytes == 2 && ((out->start != nullptr) == (out->finish != nullptr));
+  if (!pe::plan_global(g, K, flags, allow_compact, &p)) return PE_ERR_UNSUPPORTED;
   if (p.workspace > (size_t)PE_NOALLOC_SCRATCH_BYTES) return PE_ERR_SCRATCH_LIMIT;
   if (K == 0) return PE_OK;
   if (!assign || !order) return PE_ERR_INVALID_ARG;

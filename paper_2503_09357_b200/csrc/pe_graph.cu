@@ -136,6 +136,58 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
   int32_t* cap = (int32_t*)(blob.data() + lay.cap);
   for (int32_t j = 0; j < D; ++j) cap[j] = d->mem_capacity ? d->mem_capacity[j] : INT32_MAX;
 
+  // compact encoding, when every value fits its field
+  bool no_channel = false;
+  if (d->link_class)
+    for (int32_t a = 0; a < D * D; ++a) no_channel = no_channel || d->link_class[a] == 0xFF;
+  bool narrow = V <= 65535 && L <= 2 && mdeg <= 255 && E < (1 << 24);
+  for (int32_t i = 0; narrow && i < V; ++i)
+    narrow = ops[i].dur <= 65535 && ops[i].mem_delta >= -32768 && ops[i].mem_delta <= 32767;
+  for (int64_t q = 0; narrow && q < (int64_t)E * L; ++q) narrow = comm[q] <= 65535;
+  std::vector<uint8_t> nblob;
+  g->narrow_ok = narrow;
+  g->d_nblob = nullptr;
+  std::memset(&g->nview, 0, sizeof(g->nview));
+  if (narrow) {
+    PeNarrowView& nv = g->nview;
+    nv.V = V; nv.E = E; nv.D = D; nv.L = L;
+    nv.has_weight = g->has_weight ? 1 : 0;
+    nv.need_cls = (L > 1 || no_channel) ? 1 : 0;
+    uint64_t nat = 0;
+    nv.ops = (uint32_t)nat;    nat = align16(nat + (uint64_t)V * 16);
+    nv.edges = (uint32_t)nat;  nat = align16(nat + (uint64_t)E * 4 * L);
+    nv.weight = (uint32_t)nat; nat = align16(nat + (g->has_weight ? (uint64_t)V * 4 : 0));
+    nv.cls = (uint32_t)nat;    nat = align16(nat + (uint64_t)D * D);
+    nv.cap = (uint32_t)nat;    nat = align16(nat + (uint64_t)D * 4);
+    nv.bytes = (uint32_t)nat;
+    nblob.assign(nv.bytes, 0);
+    uint32_t* nops = (uint32_t*)(nblob.data() + nv.ops);
+    uint32_t* nedges = (uint32_t*)(nblob.data() + nv.edges);
+    for (int32_t q = 0; q < E; ++q) {
+      const uint32_t lo = ((uint32_t)comm[(size_t)q * L] << 16) | (uint32_t)pred[q];
+      if (L == 1) nedges[q] = lo;
+      else { nedges[2 * (size_t)q] = lo; nedges[2 * (size_t)q + 1] = (uint32_t)comm[(size_t)q * L + 1]; }
+    }
+    for (int32_t i = 0; i < V; ++i) {
+      uint32_t* r = nops + 4 * (size_t)i;
+      const int32_t b = ops[i].edge_begin, n = ops[i].indeg;
+      r[0] = ((uint32_t)b << 8) | (uint32_t)n;
+      r[1] = ((uint32_t)(uint16_t)(int16_t)ops[i].mem_delta << 16) | (uint32_t)ops[i].dur;
+      // a missing inline edge points at the sentinel operator V (always "ended at 0", zero delay)
+      const uint32_t none = (uint32_t)V;
+      if (L == 1) {
+        r[2] = n > 0 ? nedges[b] : none;
+        r[3] = n > 1 ? nedges[b + 1] : none;
+      } else {
+        r[2] = n > 0 ? nedges[2 * (size_t)b] : none;
+        r[3] = n > 0 ? nedges[2 * (size_t)b + 1] : 0u;
+      }
+    }
+    if (g->has_weight) std::memcpy(nblob.data() + nv.weight, d->mem_weight, (size_t)V * 4);
+    if (d->link_class) std::memcpy(nblob.data() + nv.cls, d->link_class, (size_t)D * D);
+    std::memcpy(nblob.data() + nv.cap, cap, (size_t)D * 4);
+  }
+
   cudaDeviceProp prop;
   int prev = -1;
   bool ok = cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(cuda_device) == cudaSuccess &&
@@ -147,12 +199,16 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
          cudaMalloc((void**)&g->d_error, 256) == cudaSuccess &&
          cudaMemcpy(g->d_blob, blob.data(), lay.bytes, cudaMemcpyHostToDevice) == cudaSuccess &&
          cudaMemset(g->d_error, 0, 256) == cudaSuccess;
+    if (ok && narrow)
+      ok = cudaMalloc((void**)&g->d_nblob, nblob.size()) == cudaSuccess &&
+           cudaMemcpy(g->d_nblob, nblob.data(), nblob.size(), cudaMemcpyHostToDevice) == cudaSuccess;
   }
   if (prev >= 0) cudaSetDevice(prev);
   if (!ok) {
     cudaGetLastError();
     if (g->d_blob) cudaFree(g->d_blob);
     if (g->d_error) cudaFree(g->d_error);
+    if (g->d_nblob) cudaFree(g->d_nblob);
     delete g;
     return PE_ERR_CUDA;
   }
@@ -165,7 +221,8 @@ extern "C" int pe_destroy(pe_graph* g) {
   int prev = -1;
   cudaGetDevice(&prev);
   cudaSetDevice(g->device);
-  const bool ok = cudaFree(g->d_blob) == cudaSuccess && cudaFree(g->d_error) == cudaSuccess;
+  bool ok = cudaFree(g->d_blob) == cudaSuccess && cudaFree(g->d_error) == cudaSuccess;
+  if (g->d_nblob) ok = cudaFree(g->d_nblob) == cudaSuccess && ok;
   if (prev >= 0) cudaSetDevice(prev);
   delete g;
   return ok ? PE_OK : PE_ERR_CUDA;

@@ -34,6 +34,29 @@ struct PeGraphView {
   PeBlobLayout lay;
 };
 
+// Compact ("narrow") encoding of the same graph, built when every value fits: V <= 65535,
+// D^o and D^c below 65536, A in int16, L <= 2, in-degree <= 255, E < 2^24.  One 16-byte record
+// per operator carries its first incoming edges inline, so the common operator needs a single
+// shared-memory load:
+//   w0 = edge_begin << 8 | indeg        (CSR slot of its first incoming edge, count)
+//   w1 = (uint16)A << 16 | dur
+//   L == 1: w2, w3 = incoming edges 0 and 1 as  comm << 16 | pred
+//   L == 2: (w2, w3) = incoming edge 0 as  (comm[class 0] << 16 | pred, comm[class 1])
+// An inline slot without an edge holds pred = V with zero delay: kernels keep a sentinel state
+// row V ("ended at time 0 on machine 0"), so the slot can be evaluated without a branch.
+// followed by all incoming edges again in CSR order (4 bytes each for L == 1, 8 for L == 2).
+struct PeNarrowView {
+  int32_t V, E, D, L;
+  int32_t has_weight;
+  int32_t need_cls;   // the link-class table must be consulted (L > 1 or some pair has no channel)
+  uint32_t ops;       // uint4[V]
+  uint32_t edges;     // uint32[E] (L == 1) or uint2[E] (L == 2)
+  uint32_t weight;    // int32[V] if has_weight
+  uint32_t cls;       // uint8[D*D]
+  uint32_t cap;       // int32[D]
+  uint32_t bytes;     // total, multiple of 16
+};
+
 struct pe_graph {
   int32_t V, E, D, L;
   int device;
@@ -43,6 +66,9 @@ struct pe_graph {
   int32_t max_indeg;
   PeBlobLayout lay;
   uint8_t* d_blob;     // device copy of the blob
+  bool narrow_ok;      // the compact encoding exists
+  PeNarrowView nview;
+  uint8_t* d_nblob;    // device copy of the compact encoding (nullptr if !narrow_ok)
   int* d_error;        // device status word (0 = ok)
   int sm_count;
   size_t smem_optin;   // max dynamic shared memory per block

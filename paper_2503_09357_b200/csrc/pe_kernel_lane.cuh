@@ -1,0 +1,213 @@
+// One thread per candidate over the compact graph encoding: the kernel behind the SHARED
+// variant (STATE_SMEM = true) and the GLOBAL variant of graphs that have a compact encoding
+// (STATE_SMEM = false).
+//
+//  * per-operator state word: end time << 8 | machine; 0xFFFFFFxx until the operator is
+//    scheduled.  With by-operator assignments the machine byte is filled in by the initial
+//    pass (a coalesced read of `assign`), so the main loop never gathers from `assign`.
+//      STATE_SMEM:  shared memory, [operator][thread] - a lane's gathers stay in its own bank;
+//      otherwise:   the caller's workspace, [operator][K] candidate-interleaved.
+//    Row V is a sentinel ("ended at time 0 on machine 0"): the compact encoding points the
+//    inline edge slots of operators with fewer incoming edges at it, so those slots are
+//    evaluated without a branch and change nothing.
+//  * per-machine state: one 16-byte record {free time, busy, level, peak} per (machine,
+//    thread) in shared memory: one 128-bit load and one 128-bit store per step.
+//  * graph: compact encoding (16-byte operator record with the first incoming edges inline),
+//    staged into shared memory by bulk copy (STATE_SMEM) or read through the read-only cache.
+//  * order entries (and by-position machine ids) are fetched kUnroll positions ahead into
+//    register rings, the operator record one position ahead.
+//  * validity (order entry range, repeated operator, predecessor not scheduled, machine range)
+//    is accumulated with min/max and tested once at the end; an out-of-range entry is clamped
+//    so that indexing stays in bounds.
+// The recurrence itself (Eqs. 3, 7-8, 11-13, 16-19) is the one stated at the top of pe_eval.cu.
+#pragma once
+#include "pe_device.cuh"
+
+namespace pe {
+
+constexpr int kUnroll = 8;
+constexpr uint32_t kUnscheduled = 0xFFFFFF00u;  // state words at or above this: not scheduled yet
+
+struct NarrowPtrs {
+  const uint4* ops;
+  const uint32_t* edges;
+  const int32_t* weight;
+  const uint8_t* cls;
+  const int32_t* cap;
+};
+
+__device__ __forceinline__ NarrowPtrs narrow_ptrs(const uint8_t* base, const PeNarrowView& g) {
+  NarrowPtrs p;
+  p.ops = reinterpret_cast<const uint4*>(base + g.ops);
+  p.edges = reinterpret_cast<const uint32_t*>(base + g.edges);
+  p.weight = g.has_weight ? reinterpret_cast<const int32_t*>(base + g.weight) : nullptr;
+  p.cls = base + g.cls;
+  p.cap = reinterpret_cast<const int32_t*>(base + g.cap);
+  return p;
+}
+
+// CLS: 0 = one link class, every pair connected (no table lookup); 1 = one class, some pair
+// without a channel; 2 = two classes.  IdxT: uint32_t when (V+1)*K fits in 32 bits.
+// TIMES: start and finish are both written (true) or both absent (false).
+template <typename IdxT, bool BY_POS, int CLS, bool STATE_SMEM, bool TIMES>
+__global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const uint8_t* __restrict__ nblob, int64_t K,
+                                                           const uint8_t* __restrict__ assign,
+                                                           const uint16_t* __restrict__ order, pe_outputs out,
+                                                           uint32_t flags, int* err, uint32_t* __restrict__ gstate) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  constexpr bool TWO_CLASS = CLS == 2;
+  constexpr bool NEED_CLS = CLS != 0;
+  const int T = blockDim.x;
+  const int t = threadIdx.x;
+  const int D = g.D, V = g.V;
+  uint8_t* sm = smem_raw;
+  const uint8_t* gbase = nblob;
+  if (STATE_SMEM) {
+    uint64_t* bar = reinterpret_cast<uint64_t*>(smem_raw + g.bytes);
+    if (!stage_blob(smem_raw, nblob, g.bytes, bar, err)) return;
+    gbase = smem_raw;
+    sm = smem_raw + g.bytes + 16;
+  }
+  const NarrowPtrs gp = narrow_ptrs(gbase, g);
+  int4* dev = reinterpret_cast<int4*>(sm) + t;  // [D][T] {free, busy, level, peak}
+  int32_t* wsum = reinterpret_cast<int32_t*>(sm + (size_t)D * T * 16) + t;  // [D][T], only with weights
+  const size_t wsum_bytes = g.has_weight ? (size_t)D * T * 4 : 0;
+
+  const int64_t c = (int64_t)blockIdx.x * T + t;
+  if (c >= K) return;
+  const IdxT Ki = (IdxT)K;
+  // state word of operator p is state[p * pitch]
+  uint32_t* state = STATE_SMEM ? reinterpret_cast<uint32_t*>(sm + (size_t)D * T * 16 + wsum_bytes) + t : gstate + c;
+  const IdxT pitch = STATE_SMEM ? (IdxT)T : Ki;
+
+  const uint16_t* order_col = order + c;
+  const uint8_t* assign_col = assign + c;
+  {  // initial state: unscheduled; by-operator assignments also deposit the machine byte
+    IdxT at = 0;
+    for (int i = 0; i < V; ++i) {
+      state[(IdxT)i * pitch] = BY_POS ? 0xFFFFFFFFu : (kUnscheduled | (uint32_t)assign_col[at]);
+      at += Ki;
+    }
+    state[(IdxT)V * pitch] = 0u;
+  }
+  for (int j = 0; j < D; ++j) {
+    dev[j * T] = make_int4(0, 0, 0, 0);
+    if (gp.weight) wsum[j * T] = 0;
+  }
+  const bool by_op_times = (flags & PE_TIMES_BY_OP) != 0;
+  const uint32_t vmax = (uint32_t)(V - 1), dmax = (uint32_t)(D - 1);
+  const IdxT off_last = (IdxT)vmax * Ki;
+  uint32_t st = 0;
+  int32_t z = 0;
+  // validity accumulators, tested after the loop
+  uint32_t order_max = 0, dev_max = 0, pred_max = 0, own_min = 0xFFFFFFFFu;
+
+  int32_t* start_col = TIMES ? out.start + c : nullptr;
+  int32_t* finish_col = TIMES ? out.finish + c : nullptr;
+
+  // register rings: o0/a0 = the block being processed, o1/a1 = the block after it
+  uint32_t o0[kUnroll], o1[kUnroll], a0[kUnroll], a1[kUnroll];
+  IdxT off_load = 0;  // element offset (row * K) of the next row to prefetch, clamped to the last row
+  auto prefetch = [&](uint32_t (&od)[kUnroll], uint32_t (&ad)[kUnroll]) {
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const IdxT at = min(off_load, off_last);
+      od[u] = (uint32_t)order_col[at];
+      if (BY_POS) ad[u] = (uint32_t)assign_col[at];
+      off_load += Ki;
+    }
+  };
+  prefetch(o0, a0);
+  prefetch(o1, a1);
+  uint4 rec_next = gp.ops[min(o0[0], vmax)];
+  IdxT off_k = 0;  // element offset of the current position's row
+
+  auto step = [&](const uint32_t iu, const uint32_t a_pos, const uint32_t nxt) {
+    const uint4 rec = rec_next;
+    rec_next = gp.ops[min(nxt, vmax)];  // operator record of the next position, while this one is computed
+    order_max = max(order_max, iu);
+    const uint32_t i = min(iu, vmax);
+    const uint32_t mine = state[(IdxT)i * pitch];
+    own_min = min(own_min, mine);
+    const uint32_t jr = BY_POS ? a_pos : (mine & 0xFFu);
+    dev_max = max(dev_max, jr);
+    const int j = (int)min(jr, dmax);
+    const int4 dv = dev[j * T];
+    const int indeg = (int)(rec.x & 0xFFu);
+    const int32_t dur = (int32_t)(rec.y & 0xFFFFu);
+    const int32_t dA = (int32_t)rec.y >> 16;
+
+    // one incoming edge: lo = comm[class 0] << 16 | pred, hi = comm[class 1]
+    auto edge_time = [&](uint32_t lo, uint32_t hi) -> int32_t {
+      const uint32_t p = lo & 0xFFFFu;
+      const uint32_t w = state[(IdxT)p * pitch];
+      pred_max = max(pred_max, w);
+      const int xp = (int)(w & 0xFFu);
+      uint32_t delay = lo >> 16;
+      if (NEED_CLS) {
+        const uint32_t cl = gp.cls[xp * D + j];
+        if (TWO_CLASS) delay = cl == 1u ? hi : delay;
+        if (cl == 0xFFu) {
+          delay = 0;
+          if (p != (uint32_t)V && xp != j) st |= PE_STATUS_NO_CHANNEL;
+        }
+      }
+      return (int32_t)(w >> 8) + (xp != j ? (int32_t)delay : 0);
+    };
+    int32_t r = edge_time(rec.z, rec.w);
+    if (TWO_CLASS) {
+      if (indeg > 1) {
+        const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + (rec.x >> 8);
+        for (int q = 1; q < indeg; ++q) r = max(r, edge_time(ed[q].x, ed[q].y));
+      }
+    } else {
+      r = max(r, edge_time(rec.w, 0u));
+      if (indeg > 2) {
+        const uint32_t* ed = gp.edges + (rec.x >> 8);
+        for (int q = 2; q < indeg; ++q) r = max(r, edge_time(ed[q], 0u));
+      }
+    }
+    const int32_t s = max(r, dv.x);
+    const int32_t e = s + dur;
+    const int32_t lv = dv.z + dA;
+    dev[j * T] = make_int4(e, dv.y + dur, lv, max(dv.w, lv));
+    state[(IdxT)i * pitch] = ((uint32_t)e << 8) | (uint32_t)j;
+    if (gp.weight) wsum[j * T] += gp.weight[i];
+    z = max(z, e);
+    if (TIMES) {
+      const IdxT at = by_op_times ? (IdxT)i * Ki : off_k;
+      start_col[at] = s;
+      finish_col[at] = e;
+    }
+    off_k += Ki;
+  };
+
+  int kb = 0;
+  for (; kb + kUnroll <= V; kb += kUnroll) {
+    uint32_t o2[kUnroll], a2[kUnroll];
+    prefetch(o2, a2);
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) step(o0[u], a0[u], u + 1 < kUnroll ? o0[(u + 1) % kUnroll] : o1[0]);
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) { o0[u] = o1[u]; o1[u] = o2[u]; a0[u] = a1[u]; a1[u] = a2[u]; }
+  }
+#pragma unroll
+  for (int u = 0; u < kUnroll; ++u)  // the last, partial block
+    if (kb + u < V) step(o0[u], a0[u], o0[(u + 1) % kUnroll]);
+
+  if (order_max > vmax) st |= PE_STATUS_ORDER_INVALID;    // an entry that is no operator
+  if (own_min < kUnscheduled) st |= PE_STATUS_ORDER_INVALID;   // an operator scheduled twice
+  if (pred_max >= kUnscheduled) st |= PE_STATUS_ORDER_INVALID;  // an operator ahead of one of its predecessors
+  if (dev_max > dmax) st |= PE_STATUS_ASSIGN_RANGE;
+  for (int j = 0; j < D; ++j) {
+    const int4 dv = dev[j * T];
+    const int32_t pk = dv.w + (gp.weight ? wsum[j * T] : 0);  // the weights are resident from the start (Eq. 16)
+    if (pk > gp.cap[j]) st |= PE_STATUS_MEM_EXCEEDED;
+    if (out.busy) out.busy[(size_t)j * (size_t)K + c] = dv.y;
+    if (out.peak_mem) out.peak_mem[(size_t)j * (size_t)K + c] = pk;
+  }
+  if (out.makespan) out.makespan[c] = z;
+  if (out.status) out.status[c] = st;
+}
+
+}  // namespace pe
