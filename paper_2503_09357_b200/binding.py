@@ -186,10 +186,14 @@ class Graph:
 
     def close(self):
         if getattr(self, "handle", None):
-            pe_destroy(self.handle)
+            _lib.pe_destroy(self.handle)
             self.handle = None
 
-    __del__ = close
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:   # interpreter shutdown: the library may already be gone
+            pass
 
     def variant(self, K, flags=0) -> str:
         v = pe_eval_variant(self.handle, K, flags)

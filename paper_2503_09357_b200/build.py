@@ -7,9 +7,10 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libpe.so")
-SOURCES = ["pe_graph.cu", "pe_eval.cu"]
+SOURCES = ["pe_graph.cu", "pe_eval.cu", "pe_lane.cu", "pe_warp2.cu"]
+OBJ_DIR = os.path.join(_HERE, "_build")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "--compiler-options", "-fPIC", "-shared", "-cudart", "shared"]
+              "--compiler-options", "-fPIC", "-cudart", "shared"]
 
 
 def _stale(target, deps):
@@ -20,16 +21,28 @@ def _stale(target, deps):
 
 
 def build_libpe(force: bool = False, verbose: bool = False, extra_flags=()) -> str:
-    srcs = [os.path.join(CSRC, s) for s in SOURCES]
-    deps = srcs + [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
-    deps.append(os.path.join(_ROOT, "include", "pe.h"))
-    if force or _stale(LIB, deps):
-        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        cmd = [nvcc] + NVCC_FLAGS + list(extra_flags) + ["-I", os.path.join(_ROOT, "include"), "-I", CSRC] + srcs + ["-o", LIB]
-        if verbose:
-            cmd.insert(1, "-Xptxas=-v")
-            print(" ".join(cmd))
-        subprocess.check_call(cmd)
+    """Compile every .cu of csrc/ to an object (in parallel) and link them into libpe.so."""
+    headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
+    headers.append(os.path.join(_ROOT, "include", "pe.h"))
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    jobs, objs = [], []
+    for name in SOURCES:
+        src = os.path.join(CSRC, name)
+        obj = os.path.join(OBJ_DIR, name.replace(".cu", ".o"))
+        objs.append(obj)
+        if force or _stale(obj, [src] + headers):
+            cmd = [nvcc] + NVCC_FLAGS + list(extra_flags) + ["-I", os.path.join(_ROOT, "include"), "-I", CSRC,
+                                                              "-c", src, "-o", obj]
+            if verbose:
+                cmd.insert(1, "-Xptxas=-v")
+                print(" ".join(cmd))
+            jobs.append((name, subprocess.Popen(cmd)))
+    failed = [name for name, proc in jobs if proc.wait() != 0]
+    if failed:
+        raise RuntimeError(f"nvcc failed for {failed}")
+    if jobs or force or _stale(LIB, objs):
+        subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-cudart", "shared"] + objs + ["-o", LIB])
     return LIB
 
 

@@ -12,8 +12,8 @@
 
 #include "pe_device.cuh"
 #include "pe_graph.h"
-#include "pe_kernel_lane.cuh"
 #include "pe_kernel_warp.cuh"
+#include "pe_launch.h"
 
 namespace pe {
 
@@ -201,16 +201,6 @@ __global__ void pe_eval_shared_kernel(PeGraphView g, const uint8_t* __restrict__
 // ============================================================================================
 // Host-side planning: which variant, with what launch shape.
 // ============================================================================================
-struct Plan {
-  int variant = 0;        // PE_VARIANT_* value
-  int threads = 0;        // block size
-  size_t smem = 0;        // dynamic shared memory per block
-  bool graph_smem = false;  // graph blob staged into shared memory
-  size_t workspace = 0;   // bytes of caller workspace
-  size_t ws_x_off = 0;    // offset of the machine-state array inside the workspace (generic GLOBAL, by-pos)
-  int warp_words = 0;     // WARP: 32-bit words of shared memory per candidate
-  bool compact = false;   // SHARED / GLOBAL: the compact-graph kernel (pe_eval_lane_kernel)
-};
 
 static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -251,26 +241,28 @@ static bool plan_shared(const pe_graph* g, bool allow_compact, Plan* p) {
   return false;
 }
 
-static bool plan_warp(const pe_graph* g, Plan* p) {
+static bool plan_warp(const pe_graph* g, bool allow_compact, Plan* p) {
   if (g->time_bound >= kPackedTimeLimit) return false;
-  p->compact = false;
-  size_t words = (size_t)(g->V | 1) + (size_t)5 * g->D;
+  const bool compact = g->narrow_ok && allow_compact;
+  p->compact = compact;
+  size_t words = (size_t)(g->V + 2) + (size_t)5 * g->D;
   words |= 1;  // odd stride between candidates: the initial fill hits distinct banks
   const size_t per_warp = words * 4;
   const size_t budget = g->smem_optin;
+  const size_t blob_bytes = compact ? g->nview.bytes : g->lay.bytes;
   auto fit = [&](size_t fixed) -> int {
     if (fixed + per_warp > budget) return 0;
     const size_t n = (budget - fixed) / per_warp;
     return (int)(n > 32 ? 32 : n);
   };
   const int n_global = fit(0);
-  const int n_staged = fit((size_t)g->lay.bytes + 16);
+  const int n_staged = fit(blob_bytes + 16);
   if (n_global < 1) return false;
   const bool staged = n_staged >= (n_global < 8 ? n_global : 8);
   const int n = staged ? n_staged : n_global;
   p->variant = PE_VARIANT_WARP;
   p->threads = 32 * n;
-  p->smem = (staged ? (size_t)g->lay.bytes + 16 : 0) + (size_t)n * per_warp;
+  p->smem = (staged ? blob_bytes + 16 : 0) + (size_t)n * per_warp;
   p->graph_smem = staged;
   p->workspace = 0;
   p->ws_x_off = 0;
@@ -291,7 +283,7 @@ static bool plan_global(const pe_graph* g, int64_t K, uint32_t flags, bool allow
       p->smem = T * per;
       p->graph_smem = false;
       p->ws_x_off = 0;
-      p->workspace = round_up((size_t)(g->V + 1) * (size_t)K * 4, 256);
+      p->workspace = round_up((size_t)(g->V + 1) * (size_t)((K + 31) / 32 * 32) * 4, 256);  // tiles of 32 candidates
       p->compact = true;
       return true;
     }
@@ -317,61 +309,30 @@ static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, bool allow_co
   *p = Plan();
   const uint32_t want = flags & PE_VARIANT_MASK;
   switch (want) {
-    case PE_VARIANT_AUTO:
+    case PE_VARIANT_AUTO: {
+      // Thread-per-candidate with everything on chip wins whenever at least two warps of candidates
+      // fit in shared memory.  Beyond that the state of a candidate is too large: a warp per candidate
+      // (state still on chip) wins while several warps fit on an SM; for the largest graphs it stays
+      // ahead only when many machines keep its windows short, otherwise the global-state kernel, which
+      // is bound by random DRAM accesses but keeps thousands of candidates in flight, is faster.
       if (plan_shared(g, allow_compact, p) && p->threads >= 64) return PE_OK;
-      if (plan_global(g, K, flags, allow_compact, p) && p->compact) return PE_OK;
-      if (plan_warp(g, p)) return PE_OK;
+      Plan w, gl;
+      const bool has_w = plan_warp(g, allow_compact, &w);
+      const bool has_g = plan_global(g, K, flags, allow_compact, &gl);
+      if (has_w && (w.threads >= 4 * 32 || g->D > 16 || !has_g || !gl.compact)) { *p = w; return PE_OK; }
+      if (has_g && gl.compact) { *p = gl; return PE_OK; }
       if (plan_shared(g, allow_compact, p)) return PE_OK;
-      return plan_global(g, K, flags, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+      if (has_w) { *p = w; return PE_OK; }
+      if (has_g) { *p = gl; return PE_OK; }
+      return PE_ERR_UNSUPPORTED;
+    }
     case PE_VARIANT_GLOBAL: return plan_global(g, K, flags, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
     case PE_VARIANT_SHARED: return plan_shared(g, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
-    case PE_VARIANT_WARP: return plan_warp(g, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+    case PE_VARIANT_WARP: return plan_warp(g, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
     default: return PE_ERR_UNSUPPORTED;
   }
 }
 
-template <typename Kern>
-static bool set_smem(Kern kern, size_t bytes) {
-  return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
-}
-
-// The compact-graph kernel: state in shared memory (SHARED) or in the workspace (GLOBAL).
-template <typename IdxT, bool BY_POS, int CLS, bool STATE_SMEM>
-static int launch_compact4(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* assign, const uint16_t* order,
-                           uint32_t flags, const pe_outputs& out, uint32_t* gstate, unsigned grid,
-                           cudaStream_t stream) {
-  auto go = [&](auto kern) -> int {
-    if (!set_smem(kern, p.smem)) return PE_ERR_CUDA;
-    kern<<<grid, p.threads, p.smem, stream>>>(g->nview, g->d_nblob, K, assign, order, out, flags, g->d_error, gstate);
-    return PE_OK;
-  };
-  return out.start ? go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, true>)
-                   : go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, false>);
-}
-
-template <bool BY_POS>
-static int launch_compact(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* assign, const uint16_t* order,
-                          uint32_t flags, const pe_outputs& out, uint32_t* gstate, unsigned grid,
-                          cudaStream_t stream) {
-  const bool smem_state = p.variant == PE_VARIANT_SHARED;
-  const bool idx32 = (uint64_t)(g->V + 1) * (uint64_t)K <= 0xFFFFFFFFull;
-  const int cls = g->nview.L == 2 ? 2 : (g->nview.need_cls ? 1 : 0);
-#define PE_GO(IDX, CLS, SM) return launch_compact4<IDX, BY_POS, CLS, SM>(g, p, K, assign, order, flags, out, gstate, grid, stream)
-#define PE_GO_CLS(IDX, SM)        \
-  do {                            \
-    if (cls == 2) PE_GO(IDX, 2, SM); \
-    if (cls == 1) PE_GO(IDX, 1, SM); \
-    PE_GO(IDX, 0, SM);            \
-  } while (0)
-  if (idx32) {
-    if (smem_state) PE_GO_CLS(uint32_t, true);
-    PE_GO_CLS(uint32_t, false);
-  }
-  if (smem_state) PE_GO_CLS(uint64_t, true);
-  PE_GO_CLS(uint64_t, false);
-#undef PE_GO_CLS
-#undef PE_GO
-}
 
 template <typename OrderT, bool BY_POS>
 static int launch_typed(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* assign, const void* order,
@@ -382,8 +343,10 @@ static int launch_typed(const pe_graph* g, const Plan& p, int64_t K, const uint8
   const OrderT* ord = static_cast<const OrderT*>(order);
   if (p.compact) {
     if (sizeof(OrderT) != 2) return PE_ERR_INVALID_ARG;
-    const int rc = launch_compact<BY_POS>(g, p, K, assign, static_cast<const uint16_t*>(order), flags, out,
-                                          static_cast<uint32_t*>(workspace), grid, stream);
+    const uint16_t* ord16 = static_cast<const uint16_t*>(order);
+    uint32_t* gstate = static_cast<uint32_t*>(workspace);
+    const int rc = p.variant == PE_VARIANT_WARP ? launch_warp2(g, p, BY_POS, K, assign, ord16, flags, out, grid, stream)
+                                                : launch_lane(g, p, BY_POS, K, assign, ord16, flags, out, gstate, grid, stream);
     if (rc != PE_OK) return rc;
   } else if (p.variant == PE_VARIANT_GLOBAL) {
     int32_t* e_state = static_cast<int32_t*>(workspace);

@@ -142,7 +142,7 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
     for (int32_t a = 0; a < D * D; ++a) no_channel = no_channel || d->link_class[a] == 0xFF;
   bool narrow = V <= 65535 && L <= 2 && mdeg <= 255 && E < (1 << 24);
   for (int32_t i = 0; narrow && i < V; ++i)
-    narrow = ops[i].dur <= 65535 && ops[i].mem_delta >= -32768 && ops[i].mem_delta <= 32767;
+    narrow = ops[i].dur <= 65535 && ops[i].mem_delta >= -128 && ops[i].mem_delta <= 127;
   for (int64_t q = 0; narrow && q < (int64_t)E * L; ++q) narrow = comm[q] <= 65535;
   std::vector<uint8_t> nblob;
   g->narrow_ok = narrow;
@@ -153,6 +153,7 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
     nv.V = V; nv.E = E; nv.D = D; nv.L = L;
     nv.has_weight = g->has_weight ? 1 : 0;
     nv.need_cls = (L > 1 || no_channel) ? 1 : 0;
+    nv.max_indeg = mdeg;
     uint64_t nat = 0;
     nv.ops = (uint32_t)nat;    nat = align16(nat + (uint64_t)V * 16);
     nv.edges = (uint32_t)nat;  nat = align16(nat + (uint64_t)E * 4 * L);
@@ -171,16 +172,17 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
     for (int32_t i = 0; i < V; ++i) {
       uint32_t* r = nops + 4 * (size_t)i;
       const int32_t b = ops[i].edge_begin, n = ops[i].indeg;
-      r[0] = ((uint32_t)b << 8) | (uint32_t)n;
-      r[1] = ((uint32_t)(uint16_t)(int16_t)ops[i].mem_delta << 16) | (uint32_t)ops[i].dur;
+      r[1] = ((uint32_t)n << 24) | ((uint32_t)(uint8_t)(int8_t)ops[i].mem_delta << 16) | (uint32_t)ops[i].dur;
       // a missing inline edge points at the sentinel operator V (always "ended at 0", zero delay)
       const uint32_t none = (uint32_t)V;
       if (L == 1) {
         r[2] = n > 0 ? nedges[b] : none;
         r[3] = n > 1 ? nedges[b + 1] : none;
+        r[0] = n > 3 ? (uint32_t)b : (n > 2 ? nedges[b + 2] : none);
       } else {
         r[2] = n > 0 ? nedges[2 * (size_t)b] : none;
         r[3] = n > 0 ? nedges[2 * (size_t)b + 1] : 0u;
+        r[0] = (uint32_t)b;
       }
     }
     if (g->has_weight) std::memcpy(nblob.data() + nv.weight, d->mem_weight, (size_t)V * 4);

@@ -35,20 +35,22 @@ struct PeGraphView {
 };
 
 // Compact ("narrow") encoding of the same graph, built when every value fits: V <= 65535,
-// D^o and D^c below 65536, A in int16, L <= 2, in-degree <= 255, E < 2^24.  One 16-byte record
+// D^o and D^c below 65536, A in int8, L <= 2, in-degree <= 255, E < 2^24.  One 16-byte record
 // per operator carries its first incoming edges inline, so the common operator needs a single
-// shared-memory load:
-//   w0 = edge_begin << 8 | indeg        (CSR slot of its first incoming edge, count)
-//   w1 = (uint16)A << 16 | dur
-//   L == 1: w2, w3 = incoming edges 0 and 1 as  comm << 16 | pred
-//   L == 2: (w2, w3) = incoming edge 0 as  (comm[class 0] << 16 | pred, comm[class 1])
+// load.  An edge is  lo = comm[class 0] << 16 | pred  (plus  hi = comm[class 1]  when L == 2).
+//   w1 = indeg << 24 | (uint8)A << 16 | dur
+//   L == 1: w2, w3 = lo of incoming edges 0 and 1;
+//           w0 = lo of incoming edge 2 when indeg <= 3, else the CSR slot of the first incoming
+//           edge (edges 2.. are then read from the CSR list)
+//   L == 2: (w2, w3) = (lo, hi) of incoming edge 0; w0 = CSR slot of the first incoming edge
+// followed by all incoming edges again in CSR order (4 bytes each for L == 1, 8 for L == 2).
 // An inline slot without an edge holds pred = V with zero delay: kernels keep a sentinel state
 // row V ("ended at time 0 on machine 0"), so the slot can be evaluated without a branch.
-// followed by all incoming edges again in CSR order (4 bytes each for L == 1, 8 for L == 2).
 struct PeNarrowView {
   int32_t V, E, D, L;
   int32_t has_weight;
   int32_t need_cls;   // the link-class table must be consulted (L > 1 or some pair has no channel)
+  int32_t max_indeg;  // largest in-degree (kernels skip the third inline slot when it is <= 2)
   uint32_t ops;       // uint4[V]
   uint32_t edges;     // uint32[E] (L == 1) or uint2[E] (L == 2)
   uint32_t weight;    // int32[V] if has_weight

@@ -6,7 +6,9 @@
 //    scheduled.  With by-operator assignments the machine byte is filled in by the initial
 //    pass (a coalesced read of `assign`), so the main loop never gathers from `assign`.
 //      STATE_SMEM:  shared memory, [operator][thread] - a lane's gathers stay in its own bank;
-//      otherwise:   the caller's workspace, [operator][K] candidate-interleaved.
+//      otherwise:   the caller's workspace, in tiles of 32 candidates: [tile][operator][32].
+//                   A warp then works inside its own contiguous (V+1)*128-byte region, which
+//                   keeps its random accesses within one or two pages of address translation.
 //    Row V is a sentinel ("ended at time 0 on machine 0"): the compact encoding points the
 //    inline edge slots of operators with fewer incoming edges at it, so those slots are
 //    evaluated without a branch and change nothing.
@@ -77,24 +79,38 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
   if (c >= K) return;
   const IdxT Ki = (IdxT)K;
   // state word of operator p is state[p * pitch]
-  uint32_t* state = STATE_SMEM ? reinterpret_cast<uint32_t*>(sm + (size_t)D * T * 16 + wsum_bytes) + t : gstate + c;
-  const IdxT pitch = STATE_SMEM ? (IdxT)T : Ki;
+  uint32_t* state = STATE_SMEM ? reinterpret_cast<uint32_t*>(sm + (size_t)D * T * 16 + wsum_bytes) + t
+                               : gstate + (size_t)(c >> 5) * (size_t)(V + 1) * 32 + (c & 31);
+  const uint32_t pitch = STATE_SMEM ? (uint32_t)T : 32u;
 
   const uint16_t* order_col = order + c;
   const uint8_t* assign_col = assign + c;
-  {  // initial state: unscheduled; by-operator assignments also deposit the machine byte
+  {  // initial state: unscheduled; by-operator assignments also deposit the machine byte.  The reads of
+     // `assign` go out in batches of kInitBatch so that their latency is paid once per batch, not per row.
+    constexpr int kInitBatch = 16;
     IdxT at = 0;
-    for (int i = 0; i < V; ++i) {
-      state[(IdxT)i * pitch] = BY_POS ? 0xFFFFFFFFu : (kUnscheduled | (uint32_t)assign_col[at]);
+    int i = 0;
+    if (!BY_POS) {
+      for (; i + kInitBatch <= V; i += kInitBatch) {
+        uint32_t x[kInitBatch];
+#pragma unroll
+        for (int u = 0; u < kInitBatch; ++u) { x[u] = (uint32_t)assign_col[at]; at += Ki; }
+#pragma unroll
+        for (int u = 0; u < kInitBatch; ++u) state[(uint32_t)(i + u) * pitch] = kUnscheduled | x[u];
+      }
+    }
+    for (; i < V; ++i) {
+      state[(uint32_t)i * pitch] = BY_POS ? 0xFFFFFFFFu : (kUnscheduled | (uint32_t)assign_col[at]);
       at += Ki;
     }
-    state[(IdxT)V * pitch] = 0u;
+    state[(uint32_t)V * pitch] = 0u;
   }
   for (int j = 0; j < D; ++j) {
     dev[j * T] = make_int4(0, 0, 0, 0);
     if (gp.weight) wsum[j * T] = 0;
   }
   const bool by_op_times = (flags & PE_TIMES_BY_OP) != 0;
+  const bool deep = g.max_indeg > 2;
   const uint32_t vmax = (uint32_t)(V - 1), dmax = (uint32_t)(D - 1);
   const IdxT off_last = (IdxT)vmax * Ki;
   uint32_t st = 0;
@@ -127,20 +143,20 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
     rec_next = gp.ops[min(nxt, vmax)];  // operator record of the next position, while this one is computed
     order_max = max(order_max, iu);
     const uint32_t i = min(iu, vmax);
-    const uint32_t mine = state[(IdxT)i * pitch];
+    const uint32_t mine = state[i * pitch];
     own_min = min(own_min, mine);
     const uint32_t jr = BY_POS ? a_pos : (mine & 0xFFu);
     dev_max = max(dev_max, jr);
     const int j = (int)min(jr, dmax);
     const int4 dv = dev[j * T];
-    const int indeg = (int)(rec.x & 0xFFu);
+    const int indeg = (int)(rec.y >> 24);
     const int32_t dur = (int32_t)(rec.y & 0xFFFFu);
-    const int32_t dA = (int32_t)rec.y >> 16;
+    const int32_t dA = (int32_t)(rec.y << 8) >> 24;
 
     // one incoming edge: lo = comm[class 0] << 16 | pred, hi = comm[class 1]
     auto edge_time = [&](uint32_t lo, uint32_t hi) -> int32_t {
       const uint32_t p = lo & 0xFFFFu;
-      const uint32_t w = state[(IdxT)p * pitch];
+      const uint32_t w = state[p * pitch];
       pred_max = max(pred_max, w);
       const int xp = (int)(w & 0xFFu);
       uint32_t delay = lo >> 16;
@@ -157,21 +173,24 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
     int32_t r = edge_time(rec.z, rec.w);
     if (TWO_CLASS) {
       if (indeg > 1) {
-        const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + (rec.x >> 8);
+        const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
         for (int q = 1; q < indeg; ++q) r = max(r, edge_time(ed[q].x, ed[q].y));
       }
     } else {
       r = max(r, edge_time(rec.w, 0u));
-      if (indeg > 2) {
-        const uint32_t* ed = gp.edges + (rec.x >> 8);
-        for (int q = 2; q < indeg; ++q) r = max(r, edge_time(ed[q], 0u));
+      if (deep) {  // some operator has more than two incoming edges: third inline slot, then the CSR list
+        r = max(r, edge_time(indeg > 3 ? (uint32_t)V : rec.x, 0u));
+        if (indeg > 3) {
+          const uint32_t* ed = gp.edges + rec.x;
+          for (int q = 2; q < indeg; ++q) r = max(r, edge_time(ed[q], 0u));
+        }
       }
     }
     const int32_t s = max(r, dv.x);
     const int32_t e = s + dur;
     const int32_t lv = dv.z + dA;
     dev[j * T] = make_int4(e, dv.y + dur, lv, max(dv.w, lv));
-    state[(IdxT)i * pitch] = ((uint32_t)e << 8) | (uint32_t)j;
+    state[i * pitch] = ((uint32_t)e << 8) | (uint32_t)j;
     if (gp.weight) wsum[j * T] += gp.weight[i];
     z = max(z, e);
     if (TIMES) {

@@ -1,0 +1,260 @@
+// Variant WARP over the compact graph encoding: one warp per candidate, a window of 32
+// consecutive positions of the priority order at a time, per-operator state in shared memory.
+//
+// A candidate whose state (4 bytes per operator) is too large for a thread-per-candidate
+// block still fits on chip when a whole warp shares it.  Inside a window the only things an
+// operator can wait for are (a) a predecessor that sits in the same window and (b) the
+// previous operator of its machine in the same window (Eqs. 7-8); both sit at lower lanes
+// because the order is topological.  The window is therefore resolved in rounds:
+//   set-up   each lane marks its operator "in this window, lane l" in the state, then scans
+//            its incoming edges once to find which lower lanes it depends on (`need`);
+//   rounds   a lane whose `need` lanes have all finished evaluates its operator exactly as
+//            the thread-per-candidate kernels do (ready time from the predecessors' end
+//            times plus cross-machine delays, Eqs. 11-13; start after the machine's previous
+//            operator; end = start + duration, Eq. 3) and publishes the result;
+// the lowest unfinished lane is always ready, so the rounds end after at most 32 steps.
+// Memory levels (Eqs. 16-19) do not depend on times: they are prefix sums along each
+// machine's lanes, formed once per window with shuffles.
+//
+// State word: end << 8 | machine when scheduled (end < 0xFFFF00); 0xFFFFC000 | lane << 8 |
+// machine while in the current window; 0xFFFFFF00 | machine before that.  Row V is the
+// sentinel the compact encoding's empty edge slots point at (scheduled, end 0, machine 0).
+#pragma once
+#include "pe_device.cuh"
+#include "pe_kernel_lane.cuh"
+
+namespace pe {
+
+constexpr uint32_t kDoneLimit = 0xFFFF0000u;    // state words below this carry an end time
+constexpr uint32_t kInWindow = 0xFFFFC000u;     // | lane << 8 | machine
+constexpr uint32_t kInWindowEnd = 0xFFFFE000u;
+
+template <typename IdxT, bool BY_POS, int CLS, bool GRAPH_SMEM, bool TIMES>
+__global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, const uint8_t* __restrict__ nblob, int64_t K,
+                                                             const uint8_t* __restrict__ assign,
+                                                             const uint16_t* __restrict__ order, pe_outputs out,
+                                                             uint32_t flags, int* err, int warp_words) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  constexpr uint32_t FULL = 0xFFFFFFFFu;
+  constexpr bool TWO_CLASS = CLS == 2;
+  constexpr bool NEED_CLS = CLS != 0;
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int nwarps = blockDim.x >> 5;
+  const int D = g.D, V = g.V;
+  uint8_t* sm = smem_raw;
+  const uint8_t* gbase = nblob;
+  if (GRAPH_SMEM) {
+    uint64_t* bar = reinterpret_cast<uint64_t*>(sm + g.bytes);
+    if (!stage_blob(sm, nblob, g.bytes, bar, err)) return;
+    gbase = sm;
+    sm += g.bytes + 16;
+  }
+  const NarrowPtrs gp = narrow_ptrs(gbase, g);
+  const IdxT Ki = (IdxT)K;
+  const int64_t c0 = (int64_t)blockIdx.x * nwarps;
+
+  // ---- initial state of every candidate of the block ----
+  uint32_t* all_words = reinterpret_cast<uint32_t*>(sm);
+  if (BY_POS) {
+    for (int idx = threadIdx.x; idx < nwarps * warp_words; idx += blockDim.x) all_words[idx] = 0xFFFFFFFFu;
+  } else {
+    // machine of every operator from the by-operator assignment: row i holds nwarps adjacent bytes
+    for (int idx = threadIdx.x; idx < V * nwarps; idx += blockDim.x) {
+      const int i = idx / nwarps, w = idx - i * nwarps;
+      const int64_t cc = c0 + w;
+      all_words[(size_t)w * warp_words + i] = kUnscheduled | (cc < K ? (uint32_t)assign[(size_t)i * (size_t)K + cc] : 0u);
+    }
+  }
+  __syncthreads();
+  uint32_t* state = all_words + (size_t)warp * warp_words;  // [V + 1]
+  int32_t* free_at = reinterpret_cast<int32_t*>(state + V + 1);
+  int32_t* lvl = free_at + D;
+  int32_t* peak = lvl + D;
+  int32_t* busy = peak + D;
+  int32_t* wsum = busy + D;
+  for (int j = lane; j < (gp.weight ? 5 : 4) * D; j += 32) free_at[j] = 0;
+  if (lane == 0) state[V] = 0u;
+  __syncwarp();
+
+  const int64_t c = c0 + warp;
+  if (c >= K) return;
+  const bool by_op_times = (flags & PE_TIMES_BY_OP) != 0;
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  const uint32_t vmax = (uint32_t)(V - 1), dmax = (uint32_t)(D - 1);
+  uint32_t st = 0;
+  int32_t z = 0;
+  uint32_t order_max = 0, dev_max = 0;
+  const uint16_t* order_col = order + c;
+  const uint8_t* assign_col = assign + c;
+  int32_t* start_col = TIMES ? out.start + c : nullptr;
+  int32_t* finish_col = TIMES ? out.finish + c : nullptr;
+
+  // prefetch rings: order entries (and by-position machine ids) four windows ahead, operator
+  // records two windows ahead, so that with a handful of warps per SM the window in hand never
+  // waits for global memory
+  auto load_order = [&](int k) -> uint32_t { return k < V ? (uint32_t)order_col[(IdxT)k * Ki] : 0u; };
+  auto load_apos = [&](int k) -> uint32_t { return (BY_POS && k < V) ? (uint32_t)assign_col[(IdxT)k * Ki] : 0u; };
+  uint32_t o_ring[4], a_ring[4];
+#pragma unroll
+  for (int w = 0; w < 4; ++w) { o_ring[w] = load_order(32 * w + lane); a_ring[w] = load_apos(32 * w + lane); }
+  uint4 rec_ring[2];
+  rec_ring[0] = gp.ops[min(o_ring[0], vmax)];
+  rec_ring[1] = gp.ops[min(o_ring[1], vmax)];
+
+  for (int base = 0; base < V; base += 32) {
+    const int k = base + lane;
+    const bool act = k < V;
+    const uint32_t iu = o_ring[0];
+    const uint32_t a_here = a_ring[0];
+    const uint4 rec = rec_ring[0];
+#pragma unroll
+    for (int w = 0; w < 3; ++w) { o_ring[w] = o_ring[w + 1]; a_ring[w] = a_ring[w + 1]; }
+    o_ring[3] = load_order(k + 128);
+    a_ring[3] = load_apos(k + 128);
+    rec_ring[0] = rec_ring[1];
+    rec_ring[1] = gp.ops[min(o_ring[1], vmax)];
+
+    if (act) order_max = max(order_max, iu);
+    const uint32_t i = min(iu, vmax);
+    const uint32_t mine = act ? state[i] : kUnscheduled;
+    if (mine < kUnscheduled) st |= PE_STATUS_ORDER_INVALID;  // scheduled in an earlier window: a repeated operator
+    const uint32_t jr = BY_POS ? a_here : (mine & 0xFFu);
+    if (act) dev_max = max(dev_max, jr);
+    const uint32_t j = min(jr, dmax);
+    const int indeg = (int)(rec.y >> 24);
+    const int32_t dur = (int32_t)(rec.y & 0xFFFFu);
+    const int32_t dA = (int32_t)(rec.y << 8) >> 24;
+    const uint32_t third = indeg > 3 ? (uint32_t)V : rec.x;  // L == 1: third inline edge slot
+
+    if (act) state[i] = kInWindow | ((uint32_t)lane << 8) | j;
+    __syncwarp();
+    if (act && ((state[i] >> 8) & 31u) != (uint32_t)lane) st |= PE_STATUS_ORDER_INVALID;  // repeated inside this window
+
+    // previous / last operator of the same machine inside the window
+    const uint32_t same_dev = __match_any_sync(FULL, act ? j : (0x100u | lane));
+    const uint32_t below = same_dev & lt_mask;
+    const int prev = below ? 31 - __clz(below) : -1;
+    const bool last_on_dev = (same_dev >> lane) == 1u;
+    const uint32_t i_prev = __shfl_sync(FULL, i, prev < 0 ? lane : prev);
+
+    // memory level along the machine's lanes (Eqs. 17-19): level before the window + prefix sum of A
+    int32_t lv = dA;
+    {
+      uint32_t m = below;
+      while (__any_sync(FULL, m != 0)) {
+        const int src = m ? __ffs(m) - 1 : lane;
+        const int32_t a_src = __shfl_sync(FULL, dA, src);
+        if (m) { lv += a_src; m &= m - 1; }
+      }
+    }
+    if (act) {
+      lv += lvl[j];
+      atomicMax(&peak[j], lv);
+      atomicAdd(&busy[j], dur);
+      if (gp.weight) atomicAdd(&wsum[j], gp.weight[i]);
+    }
+    __syncwarp();
+    if (act && last_on_dev) lvl[j] = lv;
+
+    // which lower lanes this operator waits for
+    uint32_t need = prev >= 0 ? (1u << prev) : 0u;
+    auto scan_need = [&](uint32_t lo) {
+      const uint32_t w = state[lo & 0xFFFFu];
+      if (w >= kDoneLimit) {
+        const uint32_t l = (w >> 8) & 31u;
+        if (w < kInWindowEnd && l < (uint32_t)lane) need |= 1u << l;
+        else st |= PE_STATUS_ORDER_INVALID;  // a predecessor that is not before this operator
+      }
+    };
+    // value of one incoming edge once its source is scheduled
+    auto edge_time = [&](uint32_t lo, uint32_t hi) -> int32_t {
+      const uint32_t p = lo & 0xFFFFu;
+      const uint32_t w = state[p];
+      const uint32_t xp = w & 0xFFu;
+      uint32_t delay = lo >> 16;
+      if (NEED_CLS) {
+        const uint32_t cl = gp.cls[xp * D + j];
+        if (TWO_CLASS) delay = cl == 1u ? hi : delay;
+        if (cl == 0xFFu) {
+          delay = 0;
+          if (p != (uint32_t)V && xp != j) st |= PE_STATUS_NO_CHANNEL;
+        }
+      }
+      return w < kDoneLimit ? (int32_t)(w >> 8) + (xp != j ? (int32_t)delay : 0) : 0;
+    };
+    if (act) {
+      scan_need(rec.z);
+      if (TWO_CLASS) {
+        const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
+        for (int q = 1; q < indeg; ++q) scan_need(ed[q].x);
+      } else {
+        scan_need(rec.w);
+        scan_need(third);
+        if (indeg > 3) {
+          const uint32_t* ed = gp.edges + rec.x;
+          for (int q = 2; q < indeg; ++q) scan_need(ed[q]);
+        }
+      }
+    }
+
+    // rounds: the lowest unfinished lane never waits, so every round finishes at least one
+    bool pend = act;
+    int32_t s = 0, e = 0;
+    uint32_t pendmask;
+    while ((pendmask = __ballot_sync(FULL, pend)) != 0) {
+      if (pend && (need & pendmask) == 0) {
+        int32_t r = edge_time(rec.z, rec.w);
+        if (TWO_CLASS) {
+          const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
+          for (int q = 1; q < indeg; ++q) r = max(r, edge_time(ed[q].x, ed[q].y));
+        } else {
+          r = max(r, edge_time(rec.w, 0u));
+          r = max(r, edge_time(third, 0u));
+          if (indeg > 3) {
+            const uint32_t* ed = gp.edges + rec.x;
+            for (int q = 2; q < indeg; ++q) r = max(r, edge_time(ed[q], 0u));
+          }
+        }
+        const int32_t fr = prev < 0 ? free_at[j] : (int32_t)(state[i_prev] >> 8);
+        s = max(r, fr);
+        e = s + dur;
+        state[i] = ((uint32_t)e << 8) | j;
+        pend = false;
+      }
+      __syncwarp();
+    }
+
+    if (act) {
+      if (last_on_dev) free_at[j] = e;
+      z = max(z, e);
+      if (TIMES) {
+        const IdxT at = (IdxT)(by_op_times ? i : (uint32_t)k) * Ki;
+        start_col[at] = s;
+        finish_col[at] = e;
+      }
+    }
+    __syncwarp();
+  }
+
+  if (order_max > vmax) st |= PE_STATUS_ORDER_INVALID;
+  if (dev_max > dmax) st |= PE_STATUS_ASSIGN_RANGE;
+  for (int off = 16; off > 0; off >>= 1) {
+    z = max(z, __shfl_xor_sync(FULL, z, off));
+    st |= __shfl_xor_sync(FULL, st, off);
+  }
+  uint32_t over = 0;
+  for (int j = lane; j < D; j += 32) {
+    const int32_t pk = peak[j] + (gp.weight ? wsum[j] : 0);
+    if (pk > gp.cap[j]) over = 1;
+    if (out.busy) out.busy[(size_t)j * (size_t)K + c] = busy[j];
+    if (out.peak_mem) out.peak_mem[(size_t)j * (size_t)K + c] = pk;
+  }
+  if (__any_sync(FULL, over != 0)) st |= PE_STATUS_MEM_EXCEEDED;
+  if (lane == 0) {
+    if (out.makespan) out.makespan[c] = z;
+    if (out.status) out.status[c] = st;
+  }
+}
+
+}  // namespace pe

@@ -1,0 +1,36 @@
+// Internal: launch plan and the launchers of the compact-graph kernels (each family of
+// kernel instantiations lives in its own translation unit so that they compile in parallel).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "pe_graph.h"
+
+namespace pe {
+
+struct Plan {
+  int variant = 0;        // PE_VARIANT_* value
+  int threads = 0;        // block size
+  size_t smem = 0;        // dynamic shared memory per block
+  bool graph_smem = false;  // graph blob staged into shared memory
+  size_t workspace = 0;   // bytes of caller workspace
+  size_t ws_x_off = 0;    // offset of the machine-state array inside the workspace (generic GLOBAL, by-pos)
+  int warp_words = 0;     // WARP: 32-bit words of shared memory per candidate
+  bool compact = false;   // SHARED / GLOBAL: the compact-graph kernel (pe_eval_lane_kernel)
+};
+
+template <typename Kern>
+static bool set_smem(Kern kern, size_t bytes) {
+  return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
+}
+
+// pe_eval_lane_kernel: state in shared memory (plan variant SHARED) or in `gstate` (GLOBAL).
+int launch_lane(const pe_graph* g, const Plan& p, bool by_pos, int64_t K, const uint8_t* assign, const uint16_t* order,
+                uint32_t flags, const pe_outputs& out, uint32_t* gstate, unsigned grid, cudaStream_t stream);
+
+// pe_eval_warp2_kernel (plan variant WARP over the compact encoding).
+int launch_warp2(const pe_graph* g, const Plan& p, bool by_pos, int64_t K, const uint8_t* assign, const uint16_t* order,
+                 uint32_t flags, const pe_outputs& out, unsigned grid, cudaStream_t stream);
+
+}  // namespace pe
