@@ -273,20 +273,26 @@ static bool plan_warp(const pe_graph* g, bool allow_compact, Plan* p) {
 static bool plan_global(const pe_graph* g, int64_t K, uint32_t flags, bool allow_compact, Plan* p) {
   p->compact = false;
   if (g->narrow_ok && allow_compact && g->time_bound < kPackedTimeLimit) {
-    // compact-graph kernel with the state in the workspace; small blocks so that several fit on an SM
+    // compact-graph kernel with the state in the workspace.  Per-machine records stay in shared
+    // memory while a 128-thread block needs at most 16 KB for them; beyond that they would cap the
+    // resident candidates, so they move to the workspace too (tiles that stay in L2).
     const size_t per = (size_t)(g->has_weight ? 20 : 16) * g->D;
-    size_t T = 128;
-    while (T > 32 && T * per > 32768) T /= 2;
-    if (T * per <= g->smem_optin) {
-      p->variant = PE_VARIANT_GLOBAL;
-      p->threads = (int)T;
-      p->smem = T * per;
-      p->graph_smem = false;
+    const size_t tiles = (size_t)((K + 31) / 32);
+    const size_t state_bytes = round_up((size_t)(g->V + 1) * tiles * 32 * 4, 256);
+    p->variant = PE_VARIANT_GLOBAL;
+    p->threads = 128;
+    p->graph_smem = false;
+    p->compact = true;
+    if (128 * per <= 16384) {
+      p->smem = 128 * per;
       p->ws_x_off = 0;
-      p->workspace = round_up((size_t)(g->V + 1) * (size_t)((K + 31) / 32 * 32) * 4, 256);  // tiles of 32 candidates
-      p->compact = true;
-      return true;
+      p->workspace = state_bytes;
+    } else {
+      p->smem = 0;
+      p->ws_x_off = state_bytes;  // offset of the per-machine records
+      p->workspace = state_bytes + round_up(tiles * 32 * per, 256);
     }
+    return true;
   }
   const size_t per_thread = (size_t)20 * g->D;
   size_t T = g->smem_optin / per_thread / 32 * 32;
@@ -312,14 +318,14 @@ static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, bool allow_co
     case PE_VARIANT_AUTO: {
       // Thread-per-candidate with everything on chip wins whenever at least two warps of candidates
       // fit in shared memory.  Beyond that the state of a candidate is too large: a warp per candidate
-      // (state still on chip) wins while several warps fit on an SM; for the largest graphs it stays
-      // ahead only when many machines keep its windows short, otherwise the global-state kernel, which
-      // is bound by random DRAM accesses but keeps thousands of candidates in flight, is faster.
+      // (state still on chip) wins while at least four warps fit on an SM; for the largest graphs the
+      // global-state kernel, which is bound by random DRAM accesses but keeps thousands of candidates
+      // in flight, is faster.
       if (plan_shared(g, allow_compact, p) && p->threads >= 64) return PE_OK;
       Plan w, gl;
       const bool has_w = plan_warp(g, allow_compact, &w);
       const bool has_g = plan_global(g, K, flags, allow_compact, &gl);
-      if (has_w && (w.threads >= 4 * 32 || g->D > 16 || !has_g || !gl.compact)) { *p = w; return PE_OK; }
+      if (has_w && (w.threads >= 4 * 32 || !has_g || !gl.compact)) { *p = w; return PE_OK; }
       if (has_g && gl.compact) { *p = gl; return PE_OK; }
       if (plan_shared(g, allow_compact, p)) return PE_OK;
       if (has_w) { *p = w; return PE_OK; }

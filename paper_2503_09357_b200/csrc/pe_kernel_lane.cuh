@@ -55,7 +55,8 @@ template <typename IdxT, bool BY_POS, int CLS, bool STATE_SMEM, bool TIMES>
 __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const uint8_t* __restrict__ nblob, int64_t K,
                                                            const uint8_t* __restrict__ assign,
                                                            const uint16_t* __restrict__ order, pe_outputs out,
-                                                           uint32_t flags, int* err, uint32_t* __restrict__ gstate) {
+                                                           uint32_t flags, int* err, uint32_t* __restrict__ gstate,
+                                                           int4* __restrict__ gdev) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   constexpr bool TWO_CLASS = CLS == 2;
   constexpr bool NEED_CLS = CLS != 0;
@@ -71,11 +72,18 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
     sm = smem_raw + g.bytes + 16;
   }
   const NarrowPtrs gp = narrow_ptrs(gbase, g);
-  int4* dev = reinterpret_cast<int4*>(sm) + t;  // [D][T] {free, busy, level, peak}
-  int32_t* wsum = reinterpret_cast<int32_t*>(sm + (size_t)D * T * 16) + t;  // [D][T], only with weights
-  const size_t wsum_bytes = g.has_weight ? (size_t)D * T * 4 : 0;
-
   const int64_t c = (int64_t)blockIdx.x * T + t;
+  // per-machine records {free, busy, level, peak}: shared memory [D][T], or (global-state kernel
+  // with many machines, where shared memory would cap the number of resident candidates) the
+  // workspace in tiles [tile of 32][D][32], which stays in L2.  Weight sums follow the same way.
+  const bool dev_global = !STATE_SMEM && gdev != nullptr;
+  const uint32_t dpitch = dev_global ? 32u : (uint32_t)T;
+  int4* dev = dev_global ? gdev + (size_t)(c >> 5) * (size_t)D * 32 + (c & 31) : reinterpret_cast<int4*>(sm) + t;
+  int32_t* wsum = dev_global
+                      ? reinterpret_cast<int32_t*>(gdev + (size_t)((K + 31) >> 5) * (size_t)D * 32) +
+                            (size_t)(c >> 5) * (size_t)D * 32 + (c & 31)
+                      : reinterpret_cast<int32_t*>(sm + (size_t)D * T * 16) + t;
+  const size_t wsum_bytes = g.has_weight ? (size_t)D * T * 4 : 0;
   if (c >= K) return;
   const IdxT Ki = (IdxT)K;
   // state word of operator p is state[p * pitch]
@@ -106,8 +114,8 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
     state[(uint32_t)V * pitch] = 0u;
   }
   for (int j = 0; j < D; ++j) {
-    dev[j * T] = make_int4(0, 0, 0, 0);
-    if (gp.weight) wsum[j * T] = 0;
+    dev[j * dpitch] = make_int4(0, 0, 0, 0);
+    if (gp.weight) wsum[j * dpitch] = 0;
   }
   const bool by_op_times = (flags & PE_TIMES_BY_OP) != 0;
   const bool deep = g.max_indeg > 2;
@@ -148,7 +156,7 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
     const uint32_t jr = BY_POS ? a_pos : (mine & 0xFFu);
     dev_max = max(dev_max, jr);
     const int j = (int)min(jr, dmax);
-    const int4 dv = dev[j * T];
+    const int4 dv = dev[j * dpitch];
     const int indeg = (int)(rec.y >> 24);
     const int32_t dur = (int32_t)(rec.y & 0xFFFFu);
     const int32_t dA = (int32_t)(rec.y << 8) >> 24;
@@ -189,9 +197,9 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
     const int32_t s = max(r, dv.x);
     const int32_t e = s + dur;
     const int32_t lv = dv.z + dA;
-    dev[j * T] = make_int4(e, dv.y + dur, lv, max(dv.w, lv));
+    dev[j * dpitch] = make_int4(e, dv.y + dur, lv, max(dv.w, lv));
     state[i * pitch] = ((uint32_t)e << 8) | (uint32_t)j;
-    if (gp.weight) wsum[j * T] += gp.weight[i];
+    if (gp.weight) wsum[j * dpitch] += gp.weight[i];
     z = max(z, e);
     if (TIMES) {
       const IdxT at = by_op_times ? (IdxT)i * Ki : off_k;
@@ -219,8 +227,8 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
   if (pred_max >= kUnscheduled) st |= PE_STATUS_ORDER_INVALID;  // an operator ahead of one of its predecessors
   if (dev_max > dmax) st |= PE_STATUS_ASSIGN_RANGE;
   for (int j = 0; j < D; ++j) {
-    const int4 dv = dev[j * T];
-    const int32_t pk = dv.w + (gp.weight ? wsum[j * T] : 0);  // the weights are resident from the start (Eq. 16)
+    const int4 dv = dev[j * dpitch];
+    const int32_t pk = dv.w + (gp.weight ? wsum[j * dpitch] : 0);  // the weights are resident from the start (Eq. 16)
     if (pk > gp.cap[j]) st |= PE_STATUS_MEM_EXCEEDED;
     if (out.busy) out.busy[(size_t)j * (size_t)K + c] = dv.y;
     if (out.peak_mem) out.peak_mem[(size_t)j * (size_t)K + c] = pk;

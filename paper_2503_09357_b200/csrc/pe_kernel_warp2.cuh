@@ -6,12 +6,13 @@
 // operator can wait for are (a) a predecessor that sits in the same window and (b) the
 // previous operator of its machine in the same window (Eqs. 7-8); both sit at lower lanes
 // because the order is topological.  The window is therefore resolved in rounds:
-//   set-up   each lane marks its operator "in this window, lane l" in the state, then scans
-//            its incoming edges once to find which lower lanes it depends on (`need`);
-//   rounds   a lane whose `need` lanes have all finished evaluates its operator exactly as
-//            the thread-per-candidate kernels do (ready time from the predecessors' end
-//            times plus cross-machine delays, Eqs. 11-13; start after the machine's previous
-//            operator; end = start + duration, Eq. 3) and publishes the result;
+//   set-up   each lane marks its operator "in this window, lane l" in the state, then reads
+//            its incoming edges once: a source that is already scheduled contributes its end
+//            time plus the cross-machine delay (Eqs. 11-13) at once; a source at a lower lane
+//            of the window is remembered (operator id and delay) and its lane joins `need`,
+//            as does the lane of the machine's previous operator (Eqs. 7-8);
+//   rounds   a lane whose `need` lanes have all finished takes the maximum of what it has and
+//            the remembered sources' end times plus delays, ends D^o later (Eq. 3), publishes;
 // the lowest unfinished lane is always ready, so the rounds end after at most 32 steps.
 // Memory levels (Eqs. 16-19) do not depend on times: they are prefix sums along each
 // machine's lanes, formed once per window with shuffles.
@@ -157,20 +158,17 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
     __syncwarp();
     if (act && last_on_dev) lvl[j] = lv;
 
-    // which lower lanes this operator waits for
-    uint32_t need = prev >= 0 ? (1u << prev) : 0u;
-    auto scan_need = [&](uint32_t lo) {
-      const uint32_t w = state[lo & 0xFFFFu];
-      if (w >= kDoneLimit) {
-        const uint32_t l = (w >> 8) & 31u;
-        if (w < kInWindowEnd && l < (uint32_t)lane) need |= 1u << l;
-        else st |= PE_STATUS_ORDER_INVALID;  // a predecessor that is not before this operator
-      }
-    };
-    // value of one incoming edge once its source is scheduled
-    auto edge_time = [&](uint32_t lo, uint32_t hi) -> int32_t {
-      const uint32_t p = lo & 0xFFFFu;
-      const uint32_t w = state[p];
+    // Classify the incoming edges once.  A source that is already scheduled contributes its end
+    // time (+ delay) to r_base right away; a source that sits at a lower lane of this window becomes
+    // a "slot" (operator id | delay << 16) to be read when that lane has finished, and its lane joins
+    // `need`.  Edges beyond the inline ones that are in-window set `more`: they are re-read from the
+    // edge list at evaluation time.
+    uint32_t need = 0;
+    int32_t r_base = 0;
+    bool more = false;
+    const uint32_t none = (uint32_t)V;  // the sentinel: always "ended at 0"
+    uint32_t slot0 = none, slot1 = none, slot2 = none, slot_prev = none;
+    auto delay_of = [&](uint32_t lo, uint32_t hi, uint32_t w) -> uint32_t {
       const uint32_t xp = w & 0xFFu;
       uint32_t delay = lo >> 16;
       if (NEED_CLS) {
@@ -178,46 +176,74 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
         if (TWO_CLASS) delay = cl == 1u ? hi : delay;
         if (cl == 0xFFu) {
           delay = 0;
-          if (p != (uint32_t)V && xp != j) st |= PE_STATUS_NO_CHANNEL;
+          if ((lo & 0xFFFFu) != none && xp != j) st |= PE_STATUS_NO_CHANNEL;
         }
       }
-      return w < kDoneLimit ? (int32_t)(w >> 8) + (xp != j ? (int32_t)delay : 0) : 0;
+      return xp != j ? delay : 0u;
+    };
+    auto classify = [&](uint32_t lo, uint32_t hi, uint32_t& slot, bool inline_slot) {
+      const uint32_t p = lo & 0xFFFFu;
+      const uint32_t w = state[p];
+      const uint32_t dly = delay_of(lo, hi, w);
+      if (w < kDoneLimit) {
+        r_base = max(r_base, (int32_t)((w >> 8) + dly));
+      } else {
+        const uint32_t l = (w >> 8) & 31u;
+        if (w < kInWindowEnd && l < (uint32_t)lane) {
+          need |= 1u << l;
+          if (inline_slot) slot = p | (dly << 16);
+          else more = true;
+        } else {
+          st |= PE_STATUS_ORDER_INVALID;  // a predecessor that is not before this operator
+        }
+      }
     };
     if (act) {
-      scan_need(rec.z);
+      uint32_t unused = none;
+      classify(rec.z, rec.w, slot0, true);
       if (TWO_CLASS) {
         const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
-        for (int q = 1; q < indeg; ++q) scan_need(ed[q].x);
+        for (int q = 1; q < indeg; ++q) classify(ed[q].x, ed[q].y, unused, false);
       } else {
-        scan_need(rec.w);
-        scan_need(third);
+        classify(rec.w, 0u, slot1, true);
+        classify(third, 0u, slot2, true);
         if (indeg > 3) {
           const uint32_t* ed = gp.edges + rec.x;
-          for (int q = 2; q < indeg; ++q) scan_need(ed[q]);
+          for (int q = 2; q < indeg; ++q) classify(ed[q], 0u, unused, false);
         }
+      }
+      if (prev < 0) {
+        r_base = max(r_base, free_at[j]);
+      } else {
+        need |= 1u << prev;  // Eqs. 7-8: after the machine's previous operator
+        slot_prev = i_prev;
       }
     }
 
     // rounds: the lowest unfinished lane never waits, so every round finishes at least one
+    auto slot_time = [&](uint32_t sl) -> int32_t { return (int32_t)((state[sl & 0xFFFFu] >> 8) + (sl >> 16)); };
     bool pend = act;
     int32_t s = 0, e = 0;
     uint32_t pendmask;
     while ((pendmask = __ballot_sync(FULL, pend)) != 0) {
       if (pend && (need & pendmask) == 0) {
-        int32_t r = edge_time(rec.z, rec.w);
-        if (TWO_CLASS) {
-          const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
-          for (int q = 1; q < indeg; ++q) r = max(r, edge_time(ed[q].x, ed[q].y));
-        } else {
-          r = max(r, edge_time(rec.w, 0u));
-          r = max(r, edge_time(third, 0u));
-          if (indeg > 3) {
+        int32_t v = max(max(r_base, slot_time(slot0)), max(slot_time(slot1), max(slot_time(slot2), slot_time(slot_prev))));
+        if (more) {  // in-window sources among the edges kept in the edge list: all finished by now
+          if (TWO_CLASS) {
+            const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
+            for (int q = 1; q < indeg; ++q) {
+              const uint32_t w = state[ed[q].x & 0xFFFFu];
+              v = max(v, (int32_t)((w >> 8) + delay_of(ed[q].x, ed[q].y, w)));
+            }
+          } else {
             const uint32_t* ed = gp.edges + rec.x;
-            for (int q = 2; q < indeg; ++q) r = max(r, edge_time(ed[q], 0u));
+            for (int q = 2; q < indeg; ++q) {
+              const uint32_t w = state[ed[q] & 0xFFFFu];
+              v = max(v, (int32_t)((w >> 8) + delay_of(ed[q], 0u, w)));
+            }
           }
         }
-        const int32_t fr = prev < 0 ? free_at[j] : (int32_t)(state[i_prev] >> 8);
-        s = max(r, fr);
+        s = v;
         e = s + dur;
         state[i] = ((uint32_t)e << 8) | j;
         pend = false;

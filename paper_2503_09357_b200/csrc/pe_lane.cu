@@ -9,7 +9,12 @@ static int launch4(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* a
                    uint32_t flags, const pe_outputs& out, uint32_t* gstate, unsigned grid, cudaStream_t stream) {
   auto go = [&](auto kern) -> int {
     if (!set_smem(kern, p.smem)) return PE_ERR_CUDA;
-    kern<<<grid, p.threads, p.smem, stream>>>(g->nview, g->d_nblob, K, assign, order, out, flags, g->d_error, gstate);
+    // GLOBAL with the per-machine records in the workspace (plan.smem == 0): they follow the state tiles
+    int4* gdev = nullptr;
+    if (p.variant == PE_VARIANT_GLOBAL && p.smem == 0)
+      gdev = reinterpret_cast<int4*>(reinterpret_cast<uint8_t*>(gstate) + p.ws_x_off);
+    kern<<<grid, p.threads, p.smem, stream>>>(g->nview, g->d_nblob, K, assign, order, out, flags, g->d_error, gstate,
+                                               gdev);
     return PE_OK;
   };
   return out.start ? go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, true>)
