@@ -126,11 +126,18 @@ int pe_eval_variant(const pe_graph* g, int64_t K, uint32_t flags);
 int pe_eval_batch(pe_graph* g, int64_t K, const uint8_t* assign, const void* order, int order_bytes, uint32_t flags,
                   const pe_outputs* out, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Host-buffer form of the same call: copies `assign` and `order` from HOST memory into the caller's
- * device staging buffers, evaluates, copies every requested output back to the HOST pointers in
- * `host_out`, and synchronises the stream before returning.  `dev_assign` [V*K] u8, `dev_order`
- * [V*K*order_bytes] and `dev_out` (device pointers for exactly the members set in host_out) are
- * caller-owned staging.  Pinned host memory makes the copies asynchronous with each other. */
+/* Host-buffer form of the same call: evaluates K candidates whose inputs and outputs live in HOST
+ * memory, and synchronises the stream before returning.  The batch is processed in chunks of
+ * candidates so that the upload of one chunk, the kernel of another and the download of a third
+ * overlap (copies run on two streams owned by the graph, kernels on `cuda_stream`); pinned host
+ * memory is needed for that overlap, pageable memory still gives correct results.
+ *   host_assign / host_order   inputs, laid out as for pe_eval_batch
+ *   host_out                   HOST pointers of the outputs wanted, laid out as for pe_eval_batch
+ *   dev_assign [V*K] u8, dev_order [V*K*order_bytes], dev_out (DEVICE pointers for exactly the
+ *   members set in host_out, each of the full size)   caller-owned staging; their contents after
+ *   the call are chunk-blocked, not the [rows][K] layout, and should be treated as scratch
+ *   workspace                  as for pe_eval_batch with this K
+ * Calls on the same graph are serialised internally (they share the graph's copy streams). */
 int pe_eval_batch_host(pe_graph* g, int64_t K, const uint8_t* host_assign, const void* host_order, int order_bytes,
                        uint32_t flags, const pe_outputs* host_out, uint8_t* dev_assign, void* dev_order,
                        const pe_outputs* dev_out, void* workspace, size_t workspace_bytes, void* cuda_stream);

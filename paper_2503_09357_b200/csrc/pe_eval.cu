@@ -7,6 +7,7 @@
 // machine's memory level moves by A_i (Eqs. 16-19).  The variants differ in where the
 // per-candidate state lives and how lanes map to candidates.
 #include <atomic>
+#include <mutex>
 #include <climits>
 #include <cstdio>
 
@@ -452,30 +453,71 @@ extern "C" int pe_eval_batch_host(pe_graph* g, int64_t K, const uint8_t* host_as
   if (cudaGetDevice(&prev) != cudaSuccess) return PE_ERR_CUDA;
   if (prev != g->device && cudaSetDevice(g->device) != cudaSuccess) return PE_ERR_CUDA;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  const size_t VK = (size_t)g->V * (size_t)K, DK = (size_t)g->D * (size_t)K;
+  const size_t V = (size_t)g->V, D = (size_t)g->D, Ks = (size_t)K, ob = (size_t)order_bytes;
+  pe_outputs want = *dev_out;  // compute only what the host asked for
+  if (!host_out->start) want.start = nullptr;
+  if (!host_out->finish) want.finish = nullptr;
+  if (!host_out->makespan) want.makespan = nullptr;
+  if (!host_out->busy) want.busy = nullptr;
+  if (!host_out->peak_mem) want.peak_mem = nullptr;
+  if (!host_out->status) want.status = nullptr;
+
+  // The batch is cut into chunks of candidates.  Chunk q's inputs go up on the graph's copy-in
+  // stream, its kernel runs on the caller's stream, its outputs come down on the copy-out stream,
+  // so the uploads, the kernels and the downloads of different chunks overlap (the two copy
+  // directions use separate DMA engines).  A chunk of Kc candidates lives in the staging buffers
+  // as a dense [rows][Kc] block at element offset rows * first; the strided host side is handled
+  // by 2-D copies.
+  int nchunks = K >= 8 * 4096 ? 8 : 1;
+  const int64_t per = ((K + nchunks - 1) / nchunks + 255) / 256 * 256;
+  nchunks = (int)((K + per - 1) / per);
+  std::lock_guard<std::mutex> lock(g->host_mutex);
   int ret = PE_OK;
-  if (cudaMemcpyAsync(dev_assign, host_assign, VK, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-      cudaMemcpyAsync(dev_order, host_order, VK * (size_t)order_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
-    ret = PE_ERR_CUDA;
-  pe_outputs run = *dev_out;  // compute only what the host asked for
-  if (!host_out->start) run.start = nullptr;
-  if (!host_out->finish) run.finish = nullptr;
-  if (!host_out->makespan) run.makespan = nullptr;
-  if (!host_out->busy) run.busy = nullptr;
-  if (!host_out->peak_mem) run.peak_mem = nullptr;
-  if (!host_out->status) run.status = nullptr;
-  if (ret == PE_OK)
-    ret = pe_eval_batch(g, K, dev_assign, dev_order, order_bytes, flags, &run, workspace, workspace_bytes, cuda_stream);
-  auto back = [&](void* h, const void* d, size_t bytes) {
-    if (ret == PE_OK && h && cudaMemcpyAsync(h, d, bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) ret = PE_ERR_CUDA;
-  };
-  back(host_out->start, run.start, VK * 4);
-  back(host_out->finish, run.finish, VK * 4);
-  back(host_out->makespan, run.makespan, (size_t)K * 4);
-  back(host_out->busy, run.busy, DK * 4);
-  back(host_out->peak_mem, run.peak_mem, DK * 4);
-  back(host_out->status, run.status, (size_t)K * 4);
+  auto ok = [&](cudaError_t e) { if (e != cudaSuccess && ret == PE_OK) ret = PE_ERR_CUDA; };
+  ok(cudaEventRecord(g->ev_begin, stream));           // copies start after the caller's earlier work
+  ok(cudaStreamWaitEvent(g->copy_in, g->ev_begin, 0));
+  ok(cudaStreamWaitEvent(g->copy_out, g->ev_begin, 0));
+  for (int q = 0; q < nchunks && ret == PE_OK; ++q) {
+    const size_t first = (size_t)q * (size_t)per;
+    const size_t Kc = (size_t)(K - (int64_t)first < per ? K - (int64_t)first : per);
+    uint8_t* d_as = dev_assign + V * first;
+    uint8_t* d_or = static_cast<uint8_t*>(dev_order) + V * first * ob;
+    ok(cudaMemcpy2DAsync(d_as, Kc, host_assign + first, Ks, Kc, V, cudaMemcpyHostToDevice, g->copy_in));
+    ok(cudaMemcpy2DAsync(d_or, Kc * ob, static_cast<const uint8_t*>(host_order) + first * ob, Ks * ob, Kc * ob, V,
+                         cudaMemcpyHostToDevice, g->copy_in));
+    ok(cudaEventRecord(g->ev_in[q], g->copy_in));
+    ok(cudaStreamWaitEvent(stream, g->ev_in[q], 0));
+    pe_outputs run;
+    run.start = want.start ? want.start + V * first : nullptr;
+    run.finish = want.finish ? want.finish + V * first : nullptr;
+    run.makespan = want.makespan ? want.makespan + first : nullptr;
+    run.busy = want.busy ? want.busy + D * first : nullptr;
+    run.peak_mem = want.peak_mem ? want.peak_mem + D * first : nullptr;
+    run.status = want.status ? want.status + first : nullptr;
+    if (ret == PE_OK)
+      ret = pe_eval_batch(g, (int64_t)Kc, d_as, d_or, order_bytes, flags, &run, workspace, workspace_bytes, cuda_stream);
+    ok(cudaEventRecord(g->ev_done[q], stream));
+    ok(cudaStreamWaitEvent(g->copy_out, g->ev_done[q], 0));
+    auto back = [&](void* h, const void* d, size_t rows, size_t elem) {  // [rows][Kc] block -> columns first.. of [rows][K]
+      if (h && ret == PE_OK)
+        ok(cudaMemcpy2DAsync(static_cast<uint8_t*>(h) + first * elem, Ks * elem, d, Kc * elem, Kc * elem, rows,
+                             cudaMemcpyDeviceToHost, g->copy_out));
+    };
+    back(host_out->start, run.start, V, 4);
+    back(host_out->finish, run.finish, V, 4);
+    back(host_out->makespan, run.makespan, 1, 4);
+    back(host_out->busy, run.busy, D, 4);
+    back(host_out->peak_mem, run.peak_mem, D, 4);
+    back(host_out->status, run.status, 1, 4);
+  }
+  ok(cudaEventRecord(g->ev_end, g->copy_out));
+  ok(cudaStreamWaitEvent(stream, g->ev_end, 0));
   if (cudaStreamSynchronize(stream) != cudaSuccess && ret == PE_OK) ret = PE_ERR_CUDA;
+  if (ret != PE_OK) {  // leave nothing of this call running on the graph's own streams
+    cudaStreamSynchronize(g->copy_in);
+    cudaStreamSynchronize(g->copy_out);
+    cudaGetLastError();
+  }
   if (prev != g->device) cudaSetDevice(prev);
   return ret;
 }

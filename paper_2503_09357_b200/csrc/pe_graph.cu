@@ -204,6 +204,15 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
     if (ok && narrow)
       ok = cudaMalloc((void**)&g->d_nblob, nblob.size()) == cudaSuccess &&
            cudaMemcpy(g->d_nblob, nblob.data(), nblob.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    if (ok) {
+      ok = cudaStreamCreateWithFlags(&g->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
+           cudaStreamCreateWithFlags(&g->copy_out, cudaStreamNonBlocking) == cudaSuccess &&
+           cudaEventCreateWithFlags(&g->ev_begin, cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&g->ev_end, cudaEventDisableTiming) == cudaSuccess;
+      for (int q = 0; ok && q < pe_graph::kMaxChunks; ++q)
+        ok = cudaEventCreateWithFlags(&g->ev_in[q], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&g->ev_done[q], cudaEventDisableTiming) == cudaSuccess;
+    }
   }
   if (prev >= 0) cudaSetDevice(prev);
   if (!ok) {
@@ -211,6 +220,15 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
     if (g->d_blob) cudaFree(g->d_blob);
     if (g->d_error) cudaFree(g->d_error);
     if (g->d_nblob) cudaFree(g->d_nblob);
+    if (g->copy_in) cudaStreamDestroy(g->copy_in);
+    if (g->copy_out) cudaStreamDestroy(g->copy_out);
+    if (g->ev_begin) cudaEventDestroy(g->ev_begin);
+    if (g->ev_end) cudaEventDestroy(g->ev_end);
+    for (int q = 0; q < pe_graph::kMaxChunks; ++q) {
+      if (g->ev_in[q]) cudaEventDestroy(g->ev_in[q]);
+      if (g->ev_done[q]) cudaEventDestroy(g->ev_done[q]);
+    }
+    cudaGetLastError();
     delete g;
     return PE_ERR_CUDA;
   }
@@ -223,6 +241,11 @@ extern "C" int pe_destroy(pe_graph* g) {
   int prev = -1;
   cudaGetDevice(&prev);
   cudaSetDevice(g->device);
+  cudaStreamDestroy(g->copy_in);
+  cudaStreamDestroy(g->copy_out);
+  cudaEventDestroy(g->ev_begin);
+  cudaEventDestroy(g->ev_end);
+  for (int q = 0; q < pe_graph::kMaxChunks; ++q) { cudaEventDestroy(g->ev_in[q]); cudaEventDestroy(g->ev_done[q]); }
   bool ok = cudaFree(g->d_blob) == cudaSuccess && cudaFree(g->d_error) == cudaSuccess;
   if (g->d_nblob) ok = cudaFree(g->d_nblob) == cudaSuccess && ok;
   if (prev >= 0) cudaSetDevice(prev);

@@ -4,6 +4,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "pe.h"
 
 // One record per operator i, 16 bytes: where its incoming edges start in the by-predecessor
@@ -72,6 +74,13 @@ struct pe_graph {
   PeNarrowView nview;
   uint8_t* d_nblob;    // device copy of the compact encoding (nullptr if !narrow_ok)
   int* d_error;        // device status word (0 = ok)
+  // pe_eval_batch_host pipelines copies and kernels over candidate chunks: one stream per copy
+  // direction and one event per chunk and stage, created with the graph; `host_mutex` serialises
+  // host-buffer calls on the same graph because they share these.
+  static constexpr int kMaxChunks = 16;
+  cudaStream_t copy_in, copy_out;
+  cudaEvent_t ev_begin, ev_end, ev_in[kMaxChunks], ev_done[kMaxChunks];
+  std::mutex host_mutex;
   int sm_count;
   size_t smem_optin;   // max dynamic shared memory per block
 };

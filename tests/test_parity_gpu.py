@@ -224,6 +224,37 @@ def test_host_buffer_entry_point(pe):
         g.close()
 
 
+def test_host_buffer_entry_point_pipelined_chunks(pe):
+    """A batch large enough to be cut into chunks (ragged last chunk): uploads, kernels and downloads of
+    different chunks overlap, and every output still lands in the caller's [rows][K] host layout."""
+    import torch
+    from oracle import pe_oracle as orc
+    w = wl.make_config(1)
+    K = 40001
+    assign, order = wl.make_candidates(w, K=K)
+    g = pe.Graph(w)
+    try:
+        for flags in (0, pe.PE_ASSIGN_BY_POS | pe.PE_TIMES_BY_OP):
+            a = wl.assign_by_pos(assign, order) if flags & pe.PE_ASSIGN_BY_POS else assign
+            h_a = torch.from_numpy(a).pin_memory(); h_o = torch.from_numpy(gu.as_signed(order)).pin_memory()
+            d_a = torch.empty_like(h_a, device="cuda"); d_o = torch.empty_like(h_o, device="cuda")
+            d_out = g.alloc_outputs(K)
+            h_out = {k: torch.full(v.shape, -5, dtype=v.dtype).pin_memory() for k, v in d_out.items()}
+            ws, ws_bytes = g.alloc_workspace(K, flags)
+            before = pe.pe_kernel_launches()
+            rc = pe.pe_eval_batch_host(g.handle, K, h_a.data_ptr(), h_o.data_ptr(), 2, flags,
+                                       pe.make_outputs(**{k: v.data_ptr() for k, v in h_out.items()}),
+                                       d_a.data_ptr(), d_o.data_ptr(),
+                                       pe.make_outputs(**{k: v.data_ptr() for k, v in d_out.items()}),
+                                       ws.data_ptr(), ws_bytes, torch.cuda.current_stream().cuda_stream)
+            assert rc == pe.PE_OK and pe.pe_kernel_launches() == before + 8
+            res = {k: v.numpy() for k, v in h_out.items()}
+            res["status"] = res["status"].view(np.uint32)
+            gu.compare(res, orc.evaluate(w, a, order, flags=flags, threads=gu.CPU_THREADS), f"pipelined host call {flags}")
+    finally:
+        g.close()
+
+
 def test_bench_configuration_sampled(pe):
     """The benchmark's own launch (sweep point V=16384, D=64 at its full K) on sampled candidates:
     every output of 512 randomly chosen candidates against the oracle, plus size-independent
