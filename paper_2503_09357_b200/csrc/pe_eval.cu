@@ -242,28 +242,44 @@ static bool plan_shared(const pe_graph* g, bool allow_compact, Plan* p) {
   return false;
 }
 
-static bool plan_warp(const pe_graph* g, bool allow_compact, Plan* p) {
+static bool plan_warp(const pe_graph* g, int64_t K, uint32_t flags, bool allow_compact, Plan* p) {
   if (g->time_bound >= kPackedTimeLimit) return false;
   const bool compact = g->narrow_ok && allow_compact;
   p->compact = compact;
+  p->slab = false;
   size_t words = (size_t)(g->V + 2) + (size_t)5 * g->D;
   words |= 1;  // odd stride between candidates: the initial fill hits distinct banks
   const size_t per_warp = words * 4;
   const size_t budget = g->smem_optin;
   const size_t blob_bytes = compact ? g->nview.bytes : g->lay.bytes;
-  auto fit = [&](size_t fixed) -> int {
-    if (fixed + per_warp > budget) return 0;
-    const size_t n = (budget - fixed) / per_warp;
-    return (int)(n > 32 ? 32 : n);
+  const bool by_pos = (flags & PE_ASSIGN_BY_POS) != 0;
+  // shared tiles of the slab mode for n warps (see pe_kernel_warp2.cuh): order entries (two buffers),
+  // by-position machine ids (two buffers), start and end times
+  auto slab_bytes = [&](size_t n) -> size_t {
+    const size_t rows = 128;
+    return 2 * rows * (n + 2) * 2 + (by_pos ? ((2 * rows * (n + 4) + 3) & ~(size_t)3) : 0) + 2 * rows * (n + 1) * 4;
   };
-  const int n_global = fit(0);
-  const int n_staged = fit(blob_bytes + 16);
+  auto fit = [&](size_t fixed, bool slab) -> int {
+    for (size_t n = 32; n >= 1; --n)
+      if (fixed + n * per_warp + (slab ? slab_bytes(n) : 0) <= budget) return (int)n;
+    return 0;
+  };
+  const int n_global = fit(0, false);
+  const int n_staged = fit(blob_bytes + 16, false);
   if (n_global < 1) return false;
-  const bool staged = n_staged >= (n_global < 8 ? n_global : 8);
-  const int n = staged ? n_staged : n_global;
+  bool staged = n_staged >= (n_global < 8 ? n_global : 8);
+  int n = staged ? n_staged : n_global;
+  // Slab mode (rows read and written contiguously through shared tiles, at the price of a block
+  // barrier per 128 positions) pays off when the rows are long: with K beyond 2^19 the 32 lanes of a
+  // window touch 32 different 2 MiB pages per array, and measured throughput of the per-lane path
+  // drops by 40 %.  It needs a block wide enough to fill memory sectors.
+  if (compact && K >= ((int64_t)1 << 19)) {
+    const int ns = fit(staged ? blob_bytes + 16 : 0, true);
+    if (ns >= 16) { p->slab = true; n = ns; }
+  }
   p->variant = PE_VARIANT_WARP;
   p->threads = 32 * n;
-  p->smem = (staged ? blob_bytes + 16 : 0) + (size_t)n * per_warp;
+  p->smem = (staged ? blob_bytes + 16 : 0) + (size_t)n * per_warp + (p->slab ? slab_bytes((size_t)n) : 0);
   p->graph_smem = staged;
   p->workspace = 0;
   p->ws_x_off = 0;
@@ -324,7 +340,7 @@ static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, bool allow_co
       // in flight, is faster.
       if (plan_shared(g, allow_compact, p) && p->threads >= 64) return PE_OK;
       Plan w, gl;
-      const bool has_w = plan_warp(g, allow_compact, &w);
+      const bool has_w = plan_warp(g, K, flags, allow_compact, &w);
       const bool has_g = plan_global(g, K, flags, allow_compact, &gl);
       if (has_w && (w.threads >= 4 * 32 || !has_g || !gl.compact)) { *p = w; return PE_OK; }
       if (has_g && gl.compact) { *p = gl; return PE_OK; }
@@ -335,7 +351,7 @@ static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, bool allow_co
     }
     case PE_VARIANT_GLOBAL: return plan_global(g, K, flags, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
     case PE_VARIANT_SHARED: return plan_shared(g, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
-    case PE_VARIANT_WARP: return plan_warp(g, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+    case PE_VARIANT_WARP: return plan_warp(g, K, flags, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
     default: return PE_ERR_UNSUPPORTED;
   }
 }

@@ -30,7 +30,14 @@ constexpr uint32_t kDoneLimit = 0xFFFF0000u;    // state words below this carry 
 constexpr uint32_t kInWindow = 0xFFFFC000u;     // | lane << 8 | machine
 constexpr uint32_t kInWindowEnd = 0xFFFFE000u;
 
-template <typename IdxT, bool BY_POS, int CLS, bool GRAPH_SMEM, bool TIMES>
+// SLAB: the block's warps (adjacent candidates) move through the order in slabs of kSlab positions
+// with a block barrier between slabs; order entries (and by-position machine ids) of a slab are read
+// from global memory row by row, coalesced, into a shared tile, and start/finish times leave through
+// shared tiles the same way.  Without it every lane reads and writes its own 2..4 bytes of a
+// different row, which costs a memory transaction per lane.
+constexpr int kSlab = 128;
+
+template <typename IdxT, bool BY_POS, int CLS, bool GRAPH_SMEM, bool TIMES, bool SLAB>
 __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, const uint8_t* __restrict__ nblob, int64_t K,
                                                              const uint8_t* __restrict__ assign,
                                                              const uint16_t* __restrict__ order, pe_outputs out,
@@ -79,7 +86,8 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
   __syncwarp();
 
   const int64_t c = c0 + warp;
-  if (c >= K) return;
+  const bool cand = c < K;           // the last block may have warps without a candidate
+  if (!SLAB && !cand) return;        // (with SLAB they still take part in the tile traffic and barriers)
   const bool by_op_times = (flags & PE_TIMES_BY_OP) != 0;
   const uint32_t lt_mask = (1u << lane) - 1u;
   const uint32_t vmax = (uint32_t)(V - 1), dmax = (uint32_t)(D - 1);
@@ -91,31 +99,10 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
   int32_t* start_col = TIMES ? out.start + c : nullptr;
   int32_t* finish_col = TIMES ? out.finish + c : nullptr;
 
-  // prefetch rings: order entries (and by-position machine ids) four windows ahead, operator
-  // records two windows ahead, so that with a handful of warps per SM the window in hand never
-  // waits for global memory
-  auto load_order = [&](int k) -> uint32_t { return k < V ? (uint32_t)order_col[(IdxT)k * Ki] : 0u; };
-  auto load_apos = [&](int k) -> uint32_t { return (BY_POS && k < V) ? (uint32_t)assign_col[(IdxT)k * Ki] : 0u; };
-  uint32_t o_ring[4], a_ring[4];
-#pragma unroll
-  for (int w = 0; w < 4; ++w) { o_ring[w] = load_order(32 * w + lane); a_ring[w] = load_apos(32 * w + lane); }
-  uint4 rec_ring[2];
-  rec_ring[0] = gp.ops[min(o_ring[0], vmax)];
-  rec_ring[1] = gp.ops[min(o_ring[1], vmax)];
-
-  for (int base = 0; base < V; base += 32) {
-    const int k = base + lane;
-    const bool act = k < V;
-    const uint32_t iu = o_ring[0];
-    const uint32_t a_here = a_ring[0];
-    const uint4 rec = rec_ring[0];
-#pragma unroll
-    for (int w = 0; w < 3; ++w) { o_ring[w] = o_ring[w + 1]; a_ring[w] = a_ring[w + 1]; }
-    o_ring[3] = load_order(k + 128);
-    a_ring[3] = load_apos(k + 128);
-    rec_ring[0] = rec_ring[1];
-    rec_ring[1] = gp.ops[min(o_ring[1], vmax)];
-
+  // One window: lane l holds position k of the order (act = it exists), operator entry iu, by-position
+  // machine id a_here and the operator's record.  Returns start, end and the (clamped) operator.
+  auto window = [&](const bool act, const uint32_t iu, const uint32_t a_here, const uint4 rec, int32_t& s_out,
+                    int32_t& e_out, uint32_t& i_out) {
     if (act) order_max = max(order_max, iu);
     const uint32_t i = min(iu, vmax);
     const uint32_t mine = act ? state[i] : kUnscheduled;
@@ -251,16 +238,127 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
       __syncwarp();
     }
 
-    if (act) {
-      if (last_on_dev) free_at[j] = e;
-      z = max(z, e);
-      if (TIMES) {
+    if (act && last_on_dev) free_at[j] = e;
+    if (act) z = max(z, e);
+    s_out = s; e_out = e; i_out = i;
+    __syncwarp();
+  };
+
+  if (!SLAB) {
+    // prefetch rings: order entries (and by-position machine ids) four windows ahead, operator
+    // records two windows ahead, so that with a handful of warps per SM the window in hand never
+    // waits for global memory
+    auto load_order = [&](int k) -> uint32_t { return k < V ? (uint32_t)order_col[(IdxT)k * Ki] : 0u; };
+    auto load_apos = [&](int k) -> uint32_t { return (BY_POS && k < V) ? (uint32_t)assign_col[(IdxT)k * Ki] : 0u; };
+    uint32_t o_ring[4], a_ring[4];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) { o_ring[w] = load_order(32 * w + lane); a_ring[w] = load_apos(32 * w + lane); }
+    uint4 rec_ring[2];
+    rec_ring[0] = gp.ops[min(o_ring[0], vmax)];
+    rec_ring[1] = gp.ops[min(o_ring[1], vmax)];
+
+    for (int base = 0; base < V; base += 32) {
+      const int k = base + lane;
+      const bool act = k < V;
+      const uint32_t iu = o_ring[0];
+      const uint32_t a_here = a_ring[0];
+      const uint4 rec = rec_ring[0];
+#pragma unroll
+      for (int w = 0; w < 3; ++w) { o_ring[w] = o_ring[w + 1]; a_ring[w] = a_ring[w + 1]; }
+      o_ring[3] = load_order(k + 128);
+      a_ring[3] = load_apos(k + 128);
+      rec_ring[0] = rec_ring[1];
+      rec_ring[1] = gp.ops[min(o_ring[1], vmax)];
+      int32_t s, e;
+      uint32_t i;
+      window(act, iu, a_here, rec, s, e, i);
+      if (TIMES && act) {
         const IdxT at = (IdxT)(by_op_times ? i : (uint32_t)k) * Ki;
         start_col[at] = s;
         finish_col[at] = e;
       }
     }
-    __syncwarp();
+  } else {
+    // ---- slab mode: shared tiles behind the per-warp state ----
+    // in_tile [2][kSlab][nwarps + 2] u16, apos_tile [2][kSlab][nwarps + 4] u8 (by-position ids),
+    // s_tile / e_tile [kSlab][nwarps + 1] int32; the odd pitches keep a warp's column accesses and the
+    // block's row accesses free of bank conflicts.
+    const int in_pitch = nwarps + 2, ap_pitch = nwarps + 4, out_pitch = nwarps + 1;
+    uint16_t* in_tile = reinterpret_cast<uint16_t*>(all_words + (size_t)nwarps * warp_words);
+    uint8_t* apos_tile = reinterpret_cast<uint8_t*>(in_tile + (size_t)2 * kSlab * in_pitch);
+    int32_t* s_tile = reinterpret_cast<int32_t*>(apos_tile + (BY_POS ? (((size_t)2 * kSlab * ap_pitch + 3) & ~(size_t)3) : 0));
+    int32_t* e_tile = s_tile + (size_t)kSlab * out_pitch;
+    const int nthreads = blockDim.x;
+    constexpr int kPer = kSlab / 32;  // tile elements per thread and slab (kSlab * nwarps / (32 * nwarps))
+    const int nslabs = (V + kSlab - 1) / kSlab;
+    uint16_t o_reg[kPer];
+    uint8_t a_reg[kPer];
+    auto fetch_slab = [&](int sb) {   // rows of slab sb, coalesced: consecutive threads take consecutive candidates
+#pragma unroll
+      for (int q = 0; q < kPer; ++q) {
+        const int el = threadIdx.x + q * nthreads;
+        const int r = el / nwarps, w = el - r * nwarps;
+        const int row = sb * kSlab + r;
+        const bool ok = row < V && c0 + w < K;
+        o_reg[q] = ok ? order[(size_t)row * (size_t)K + (size_t)(c0 + w)] : (uint16_t)0;
+        if (BY_POS) a_reg[q] = ok ? assign[(size_t)row * (size_t)K + (size_t)(c0 + w)] : (uint8_t)0;
+      }
+    };
+    auto stash_slab = [&](int buf) {
+#pragma unroll
+      for (int q = 0; q < kPer; ++q) {
+        const int el = threadIdx.x + q * nthreads;
+        const int r = el / nwarps, w = el - r * nwarps;
+        in_tile[((size_t)buf * kSlab + r) * in_pitch + w] = o_reg[q];
+        if (BY_POS) apos_tile[((size_t)buf * kSlab + r) * ap_pitch + w] = a_reg[q];
+      }
+    };
+    fetch_slab(0);
+    stash_slab(0);
+    __syncthreads();
+    for (int sb = 0; sb < nslabs; ++sb) {
+      const int buf = sb & 1;
+      if (sb + 1 < nslabs) fetch_slab(sb + 1);   // in flight while this slab is computed
+      if (cand) {
+        for (int wdw = 0; wdw < kSlab / 32; ++wdw) {
+          const int r = wdw * 32 + lane;
+          const int k = sb * kSlab + r;
+          if (sb * kSlab + wdw * 32 >= V) break;   // warp-uniform
+          const bool act = k < V;
+          const uint32_t iu = in_tile[((size_t)buf * kSlab + r) * in_pitch + warp];
+          const uint32_t a_here = BY_POS ? (uint32_t)apos_tile[((size_t)buf * kSlab + r) * ap_pitch + warp] : 0u;
+          const uint4 rec = gp.ops[min(iu, vmax)];
+          int32_t s, e;
+          uint32_t i;
+          window(act, iu, a_here, rec, s, e, i);
+          if (TIMES) {
+            if (by_op_times) {
+              if (act) { start_col[(IdxT)i * Ki] = s; finish_col[(IdxT)i * Ki] = e; }
+            } else {
+              s_tile[(size_t)r * out_pitch + warp] = s;
+              e_tile[(size_t)r * out_pitch + warp] = e;
+            }
+          }
+        }
+      }
+      if (sb + 1 < nslabs) stash_slab(buf ^ 1);
+      __syncthreads();   // this slab's times are complete in the tiles, the next slab's entries are in place
+      if (TIMES && !by_op_times) {
+#pragma unroll
+        for (int q = 0; q < kPer; ++q) {
+          const int el = threadIdx.x + q * nthreads;
+          const int r = el / nwarps, w = el - r * nwarps;
+          const int row = sb * kSlab + r;
+          if (row < V && c0 + w < K) {
+            const size_t at = (size_t)row * (size_t)K + (size_t)(c0 + w);
+            out.start[at] = s_tile[(size_t)r * out_pitch + w];
+            out.finish[at] = e_tile[(size_t)r * out_pitch + w];
+          }
+        }
+        __syncthreads();   // tiles may be overwritten by the next slab
+      }
+    }
+    if (!cand) return;
   }
 
   if (order_max > vmax) st |= PE_STATUS_ORDER_INVALID;

@@ -17,7 +17,8 @@ struct Plan {
   size_t workspace = 0;   // bytes of caller workspace
   size_t ws_x_off = 0;    // offset of the machine-state array inside the workspace (generic GLOBAL, by-pos)
   int warp_words = 0;     // WARP: 32-bit words of shared memory per candidate
-  bool compact = false;   // SHARED / GLOBAL: the compact-graph kernel (pe_eval_lane_kernel)
+  bool compact = false;   // SHARED / GLOBAL / WARP: the compact-graph kernels
+  bool slab = false;      // WARP (compact): order entries and times go through shared tiles, a slab at a time
 };
 
 template <typename Kern>

@@ -13,8 +13,11 @@ static int launch4(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* a
                                                p.warp_words);
     return PE_OK;
   };
-  return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true>)
-                   : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false>);
+  if (p.slab)
+    return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, true>)
+                     : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, true>);
+  return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, false>)
+                   : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, false>);
 }
 
 template <bool BY_POS>

@@ -224,6 +224,23 @@ def test_host_buffer_entry_point(pe):
         g.close()
 
 
+@pytest.mark.parametrize("layout", ["default", "assign_by_pos", "times_by_op", "summary_only"])
+def test_warp_variant_with_long_rows_uses_shared_tiles(pe, layout):
+    """With K >= 2^19 the warp-per-candidate kernel moves order entries and times through shared tiles,
+    a slab of positions at a time (block barriers, ragged last block and last slab)."""
+    w = wl.make_config(5, V=256, D=8)
+    K = (1 << 19) + 77
+    assign, order = wl.make_candidates(w, K=K)
+    base = {"default": 0, "assign_by_pos": pe.PE_ASSIGN_BY_POS, "times_by_op": pe.PE_TIMES_BY_OP, "summary_only": 0}[layout]
+    a = wl.assign_by_pos(assign, order) if base & pe.PE_ASSIGN_BY_POS else assign
+    g = pe.Graph(w)
+    try:
+        gu.check(g, w, a, order, flags=base | pe.PE_VARIANT_WARP, want_times=layout != "summary_only",
+                 label=f"warp slab {layout}")
+    finally:
+        g.close()
+
+
 def test_host_buffer_entry_point_pipelined_chunks(pe):
     """A batch large enough to be cut into chunks (ragged last chunk): uploads, kernels and downloads of
     different chunks overlap, and every output still lands in the caller's [rows][K] host layout."""
