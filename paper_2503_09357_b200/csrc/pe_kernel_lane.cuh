@@ -51,7 +51,9 @@ __device__ __forceinline__ NarrowPtrs narrow_ptrs(const uint8_t* base, const PeN
 // CLS: 0 = one link class, every pair connected (no table lookup); 1 = one class, some pair
 // without a channel; 2 = two classes.  IdxT: uint32_t when (V+1)*K fits in 32 bits.
 // TIMES: start and finish are both written (true) or both absent (false).
-template <typename IdxT, bool BY_POS, int CLS, bool STATE_SMEM, bool TIMES>
+// DEPTH (one link class only): 3 = no operator has more than three incoming edges, so the three inline
+// slots are all there is and the step is straight-line code; 0 = general (inline slots, then the list).
+template <typename IdxT, bool BY_POS, int CLS, bool STATE_SMEM, bool TIMES, int DEPTH>
 __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const uint8_t* __restrict__ nblob, int64_t K,
                                                            const uint8_t* __restrict__ assign,
                                                            const uint16_t* __restrict__ order, pe_outputs out,
@@ -184,6 +186,8 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
         const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
         for (int q = 1; q < indeg; ++q) r = max(r, edge_time(ed[q].x, ed[q].y));
       }
+    } else if (DEPTH == 3) {
+      r = max(r, max(edge_time(rec.w, 0u), edge_time(rec.x, 0u)));
     } else {
       r = max(r, edge_time(rec.w, 0u));
       if (deep) {  // some operator has more than two incoming edges: third inline slot, then the CSR list

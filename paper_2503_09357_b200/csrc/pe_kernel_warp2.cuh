@@ -37,7 +37,9 @@ constexpr uint32_t kInWindowEnd = 0xFFFFE000u;
 // different row, which costs a memory transaction per lane.
 constexpr int kSlab = 128;
 
-template <typename IdxT, bool BY_POS, int CLS, bool GRAPH_SMEM, bool TIMES, bool SLAB>
+// FLAT: one link class and no operator with more than three incoming edges: the three inline slots are
+// all there is, so the edge-list loops (and the `more` path) drop out of the window code.
+template <typename IdxT, bool BY_POS, int CLS, bool GRAPH_SMEM, bool TIMES, bool SLAB, bool FLAT>
 __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, const uint8_t* __restrict__ nblob, int64_t K,
                                                              const uint8_t* __restrict__ assign,
                                                              const uint16_t* __restrict__ order, pe_outputs out,
@@ -113,7 +115,7 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
     const int indeg = (int)(rec.y >> 24);
     const int32_t dur = (int32_t)(rec.y & 0xFFFFu);
     const int32_t dA = (int32_t)(rec.y << 8) >> 24;
-    const uint32_t third = indeg > 3 ? (uint32_t)V : rec.x;  // L == 1: third inline edge slot
+    const uint32_t third = (!FLAT && indeg > 3) ? (uint32_t)V : rec.x;  // L == 1: third inline edge slot
 
     if (act) state[i] = kInWindow | ((uint32_t)lane << 8) | j;
     __syncwarp();
@@ -194,7 +196,7 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
       } else {
         classify(rec.w, 0u, slot1, true);
         classify(third, 0u, slot2, true);
-        if (indeg > 3) {
+        if (!FLAT && indeg > 3) {
           const uint32_t* ed = gp.edges + rec.x;
           for (int q = 2; q < indeg; ++q) classify(ed[q], 0u, unused, false);
         }
@@ -215,7 +217,7 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
     while ((pendmask = __ballot_sync(FULL, pend)) != 0) {
       if (pend && (need & pendmask) == 0) {
         int32_t v = max(max(r_base, slot_time(slot0)), max(slot_time(slot1), max(slot_time(slot2), slot_time(slot_prev))));
-        if (more) {  // in-window sources among the edges kept in the edge list: all finished by now
+        if (!FLAT && more) {  // in-window sources among the edges kept in the edge list: all finished by now
           if (TWO_CLASS) {
             const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
             for (int q = 1; q < indeg; ++q) {

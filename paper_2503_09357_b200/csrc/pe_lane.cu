@@ -4,7 +4,7 @@
 
 namespace pe {
 
-template <typename IdxT, bool BY_POS, int CLS, bool STATE_SMEM>
+template <typename IdxT, bool BY_POS, int CLS, bool STATE_SMEM, int DEPTH>
 static int launch4(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* assign, const uint16_t* order,
                    uint32_t flags, const pe_outputs& out, uint32_t* gstate, unsigned grid, cudaStream_t stream) {
   auto go = [&](auto kern) -> int {
@@ -17,8 +17,8 @@ static int launch4(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* a
                                                gdev);
     return PE_OK;
   };
-  return out.start ? go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, true>)
-                   : go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, false>);
+  return out.start ? go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, true, DEPTH>)
+                   : go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, false, DEPTH>);
 }
 
 template <bool BY_POS>
@@ -27,12 +27,18 @@ static int launch1(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* a
   const bool smem_state = p.variant == PE_VARIANT_SHARED;
   const bool idx32 = (uint64_t)(g->V + 1) * (uint64_t)K <= 0xFFFFFFFFull;
   const int cls = g->nview.L == 2 ? 2 : (g->nview.need_cls ? 1 : 0);
-#define PE_GO(IDX, CLS, SM) return launch4<IDX, BY_POS, CLS, SM>(g, p, K, assign, order, flags, out, gstate, grid, stream)
-#define PE_GO_CLS(IDX, SM)           \
-  do {                               \
-    if (cls == 2) PE_GO(IDX, 2, SM); \
-    if (cls == 1) PE_GO(IDX, 1, SM); \
-    PE_GO(IDX, 0, SM);               \
+  // straight-line specialisation: one fully connected link class and exactly three inline edge slots in
+  // use (measured 1.25x on the random layered graphs; for graphs with at most two incoming edges the
+  // general code, which skips the third slot by a uniform branch, is the faster one)
+  const int depth = (cls == 0 && g->max_indeg == 3) ? 3 : 0;
+#define PE_GO(IDX, CLS, SM, DEPTH) \
+  return launch4<IDX, BY_POS, CLS, SM, DEPTH>(g, p, K, assign, order, flags, out, gstate, grid, stream)
+#define PE_GO_CLS(IDX, SM)                             \
+  do {                                                 \
+    if (cls == 2) PE_GO(IDX, 2, SM, 0);                \
+    if (cls == 1) PE_GO(IDX, 1, SM, 0);                \
+    if (depth == 3) PE_GO(IDX, 0, SM, 3);              \
+    PE_GO(IDX, 0, SM, 0);                              \
   } while (0)
   if (idx32) {
     if (smem_state) PE_GO_CLS(uint32_t, true);

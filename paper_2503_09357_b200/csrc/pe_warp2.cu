@@ -13,11 +13,20 @@ static int launch4(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* a
                                                p.warp_words);
     return PE_OK;
   };
+  constexpr bool kCanFlat = CLS == 0;
+  const bool flat = kCanFlat && g->max_indeg <= 3;
+  if (flat) {
+    if (p.slab)
+      return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, true, kCanFlat>)
+                       : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, true, kCanFlat>);
+    return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, false, kCanFlat>)
+                     : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, false, kCanFlat>);
+  }
   if (p.slab)
-    return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, true>)
-                     : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, true>);
-  return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, false>)
-                   : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, false>);
+    return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, true, false>)
+                     : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, true, false>);
+  return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, false, false>)
+                   : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, false, false>);
 }
 
 template <bool BY_POS>
