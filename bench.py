@@ -373,8 +373,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--all-workloads", action="store_true",
-                    help="also time every other configuration (device-resident) and list them in other_workloads")
+    ap.add_argument("--headline-only", dest="all_workloads", action="store_false",
+                    help="skip the device-resident timing of every other configuration (other_workloads); "
+                         "it runs by default on 1 GPU and adds about a minute")
+    ap.add_argument("--all-workloads", dest="all_workloads", action="store_true", help=argparse.SUPPRESS)
+    ap.set_defaults(all_workloads=True)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
