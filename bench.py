@@ -44,7 +44,8 @@ KERNEL_OF_VARIANT = {"shared": "pe_eval_lane_kernel<STATE_SMEM=true>", "global":
 # evaluation kernel from an ncu capture, keyed by kernel variant, valid only for the kernel
 # source whose hash is recorded with it.  Reported as null when the source has changed.
 NCU_TRAFFIC = {
-    # variant: (sha256 of csrc/pe_eval.cu at capture time, bytes per op-eval, captured workload)
+    # variant: (hash of csrc/ at capture time, DRAM bytes per operator-evaluation, captured workload)
+    "global": ("0422252154d12689", 371.0, "random_layered_V16384_D64 at K = 32768 (half size), scaled by operator-evaluations"),
 }
 
 
