@@ -173,6 +173,19 @@ int pe_eval_batch_host(pe_graph* g, int64_t K, const uint8_t* host_assign, const
 int pe_eval_batch_noalloc(pe_graph* g, int64_t K, const uint8_t* assign, const void* order, int order_bytes,
                           uint32_t flags, const pe_outputs* out, void* cuda_stream);
 
+/* Selection step after an evaluation (Eq. 1: the objective is the makespan; Section III: only
+ * arrangements within every machine's memory limit are valid): among K evaluated candidates find the
+ * one with the smallest makespan whose status has none of the bits in `reject_mask` set
+ * (pass ~0u to require status == 0).  Ties go to the smallest candidate index.
+ *   makespan, status   device, [K], as written by pe_eval_batch
+ *   result             device, 4 x int64, 8-byte aligned: {best candidate index or -1 if none qualifies,
+ *                      its makespan (INT32_MAX if none), number of qualifying candidates, internal}
+ * Asynchronous on `cuda_stream`; `result` is overwritten (no initialisation needed; it also serves as
+ * the reduction's running state, so concurrent calls need separate result buffers).  K = 0 writes
+ * {-1, INT32_MAX, 0}.  K must be below 2^32. */
+int pe_select_best(int64_t K, const int32_t* makespan, const uint32_t* status, uint32_t reject_mask, int64_t* result,
+                   void* cuda_stream);
+
 /* Synchronise `cuda_stream` and return the graph's device-side error word: PE_OK, or
  * PE_ERR_TIMEOUT if a kernel gave up a bounded wait (its outputs are then invalid).  Clears the word. */
 int pe_graph_poll_error(pe_graph* g, void* cuda_stream);

@@ -94,3 +94,17 @@ def evaluate(w, assign, order, flags=0, want_times=True, threads=1, c_range=None
         with ThreadPoolExecutor(threads) as pool:
             list(pool.map(lambda t: run(cuts[t], cuts[t + 1]), range(threads)))
     return out
+
+
+def select_best(makespan, status, reject_mask=0xFFFFFFFF):
+    """The selection step written out: among candidates whose status has none of the `reject_mask`
+    bits, the smallest makespan (Eq. 1), ties to the smallest index.  Returns (index or -1,
+    makespan or INT32_MAX, number of qualifying candidates)."""
+    best, best_c, count = 2 ** 31 - 1, -1, 0
+    for c in range(len(makespan)):
+        if int(status[c]) & reject_mask:
+            continue
+        count += 1
+        if best_c < 0 or int(makespan[c]) < best:
+            best, best_c = int(makespan[c]), c
+    return best_c, best, count

@@ -63,6 +63,8 @@ _lib.pe_eval_batch_host.argtypes = [_P, ctypes.c_int64, _P, _P, ctypes.c_int, ct
 _lib.pe_eval_batch_noalloc.restype = ctypes.c_int
 _lib.pe_eval_batch_noalloc.argtypes = [_P, ctypes.c_int64, _P, _P, ctypes.c_int, ctypes.c_uint32,
                                        ctypes.POINTER(pe_outputs), _P]
+_lib.pe_select_best.restype = ctypes.c_int
+_lib.pe_select_best.argtypes = [ctypes.c_int64, _P, _P, ctypes.c_uint32, _P, _P]
 _lib.pe_graph_poll_error.restype = ctypes.c_int
 _lib.pe_graph_poll_error.argtypes = [_P, _P]
 _lib.pe_kernel_launches.restype = ctypes.c_int64
@@ -167,6 +169,12 @@ def pe_eval_batch_noalloc(handle, K, assign_ptr, order_ptr, order_bytes, flags, 
                                       int(flags), ctypes.byref(outputs), stream or None)
 
 
+def pe_select_best(K, makespan_ptr, status_ptr, reject_mask, result_ptr, stream=0) -> int:
+    """Raw call: arg-min of the makespan over the candidates whose status passes the mask (device pointers)."""
+    return _lib.pe_select_best(int(K), makespan_ptr or None, status_ptr or None, int(reject_mask) & 0xFFFFFFFF,
+                               result_ptr, stream or None)
+
+
 def pe_graph_poll_error(handle, stream=0) -> int:
     return _lib.pe_graph_poll_error(handle, stream or None)
 
@@ -217,6 +225,18 @@ class Graph:
         import torch
         n = pe_workspace_bytes(self.handle, K, flags)
         return torch.empty(max(n, 256), dtype=torch.uint8, device=torch.device("cuda", self.device)), n
+
+    def select_best(self, out, reject_mask=0xFFFFFFFF, stream=None):
+        """Index, makespan and count of the best qualifying candidate of an eval_batch result (host ints)."""
+        import torch
+        res = torch.empty(4, dtype=torch.int64, device=out["makespan"].device)
+        s = torch.cuda.current_stream(self.device).cuda_stream if stream is None else stream
+        rc = pe_select_best(out["makespan"].numel(), out["makespan"].data_ptr(), out["status"].data_ptr(), reject_mask,
+                            res.data_ptr(), s)
+        if rc != PE_OK:
+            raise PeError(rc, "pe_select_best")
+        idx, mk, cnt, _ = res.tolist()
+        return idx, mk, cnt
 
     def eval_batch(self, assign, order, flags=0, out=None, workspace=None, want_times=True, stream=None):
         """assign: cuda uint8 [V, K]; order: cuda int16/int32 [V, K] holding u16/u32 bits.

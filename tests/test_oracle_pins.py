@@ -348,3 +348,13 @@ def test_pins_reject_plausible_mistakes():
     ck.check_feasible(w, [0, 1], [0, 1], s, e)
     with pytest.raises(AssertionError):
         ck.check_left_shifted(w, [0, 1], [0, 1], s, e)
+
+
+# ---- selection step: hand cases ----
+def test_select_best_hand_cases():
+    assert orc.select_best([5, 3, 9, 3], [0, 0, 0, 0]) == (1, 3, 4)                  # tie -> smallest index
+    assert orc.select_best([5, 3, 9, 3], [0, 4, 0, 4]) == (0, 5, 2)                  # infeasible ones skipped
+    assert orc.select_best([5, 3, 9, 3], [0, 4, 0, 4], reject_mask=3) == (1, 3, 4)   # only the validity bits reject
+    assert orc.select_best([5, 3], [2, 1]) == (-1, 2 ** 31 - 1, 0)
+    assert orc.select_best([], []) == (-1, 2 ** 31 - 1, 0)
+    assert orc.select_best([7], [8], reject_mask=4) == (0, 7, 1)

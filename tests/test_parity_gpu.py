@@ -272,6 +272,40 @@ def test_host_buffer_entry_point_pipelined_chunks(pe):
         g.close()
 
 
+def test_select_best_matches_the_definition(pe):
+    import torch
+    from oracle import pe_oracle as orc
+    w = wl.make_config(1)                                   # capacity 8: a mix of feasible and infeasible candidates
+    K = 5000
+    assign, order = wl.make_candidates(w, K=K)
+    g = pe.Graph(w)
+    try:
+        out = g.eval_batch(torch.from_numpy(assign).cuda(), torch.from_numpy(gu.as_signed(order)).cuda())
+        torch.cuda.synchronize()
+        mk = out["makespan"].cpu().numpy(); st = out["status"].cpu().numpy().view(np.uint32)
+        assert (st != 0).any() and (st == 0).any()
+        for mask in (0xFFFFFFFF, 3, 4):
+            assert g.select_best(out, mask) == orc.select_best(mk, st, mask)
+        out["status"].fill_(4)                              # nobody qualifies
+        assert g.select_best(out) == (-1, 2 ** 31 - 1, 0)
+        out["status"].zero_(); out["makespan"].fill_(77)    # all tie: the first wins
+        assert g.select_best(out) == (0, 77, K)
+        res = torch.empty(4, dtype=torch.int64, device="cuda")
+        assert pe.pe_select_best(0, 0, 0, 0xFFFFFFFF, res.data_ptr(), 0) == pe.PE_OK
+        torch.cuda.synchronize()
+        assert res[:3].tolist() == [-1, 2 ** 31 - 1, 0]
+        # a batch larger than one pass of the grid
+        big_m = torch.randint(100, 1 << 20, (1 << 21,), dtype=torch.int32, device="cuda")
+        big_s = (torch.rand(1 << 21, device="cuda") < 0.5).to(torch.int32) * 4
+        got = g.select_best({"makespan": big_m, "status": big_s})
+        ok = big_s == 0
+        best = int(big_m[ok].min())
+        first = int(torch.nonzero(ok & (big_m == best))[0])
+        assert got == (first, best, int(ok.sum()))
+    finally:
+        g.close()
+
+
 def test_bench_configuration_sampled(pe):
     """The benchmark's own launch (sweep point V=16384, D=64 at its full K) on sampled candidates:
     every output of 512 randomly chosen candidates against the oracle, plus size-independent
