@@ -49,10 +49,15 @@ NCU_TRAFFIC = {
 }
 
 
+EVAL_SOURCES = ("pe_device.cuh", "pe_eval.cu", "pe_graph.cu", "pe_graph.h", "pe_kernel_lane.cuh", "pe_kernel_warp.cuh",
+                "pe_kernel_warp2.cuh", "pe_lane.cu", "pe_launch.h", "pe_warp2.cu")
+
+
 def kernel_source_hash():
+    """Hash of the sources the evaluation kernels are built from."""
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2503_09357_b200", "csrc")
-    for name in sorted(os.listdir(csrc)):
+    for name in EVAL_SOURCES:
         with open(os.path.join(csrc, name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()[:16]
