@@ -212,8 +212,12 @@ static bool plan_shared(const pe_graph* g, bool allow_compact, Plan* p) {
     const size_t per = (size_t)4 * (g->V + 1) + (size_t)(g->has_weight ? 20 : 16) * g->D;
     const size_t fixed = (size_t)g->nview.bytes + 16;
     if (fixed + 32 * per <= g->smem_optin) {
-      size_t T = (g->smem_optin - fixed) / per / 32 * 32;
+      // A block size that is a multiple of 32 keeps every lane's state column in its own bank.  That is
+      // given up only where rounding down would idle more than a sixth of the candidates that fit:
+      // with one or two warps per SM the kernel is bound by latency, not by bank conflicts.
+      size_t T = (g->smem_optin - fixed) / per;
       if (T > 256) T = 256;
+      if (T / 32 * 32 * 6 >= T * 5) T = T / 32 * 32;
       p->variant = PE_VARIANT_SHARED;
       p->threads = (int)T;
       p->smem = fixed + T * per;
@@ -333,12 +337,13 @@ static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, bool allow_co
   const uint32_t want = flags & PE_VARIANT_MASK;
   switch (want) {
     case PE_VARIANT_AUTO: {
-      // Thread-per-candidate with everything on chip wins whenever at least two warps of candidates
-      // fit in shared memory.  Beyond that the state of a candidate is too large: a warp per candidate
-      // (state still on chip) wins while at least four warps fit on an SM; for the largest graphs the
-      // global-state kernel, which is bound by random DRAM accesses but keeps thousands of candidates
-      // in flight, is faster.
-      if (plan_shared(g, allow_compact, p) && p->threads >= 64) return PE_OK;
+      // Thread-per-candidate with everything on chip wins whenever about a warp and a half of
+      // candidates fit in shared memory (measured: 55 candidates per SM at V = 1024 beat the
+      // warp-per-candidate kernel by 1.35x, 44 did not).  Beyond that the state of a candidate is too
+      // large: a warp per candidate (state still on chip) wins while at least four warps fit on an SM;
+      // for the largest graphs the global-state kernel, which is bound by random DRAM accesses but
+      // keeps thousands of candidates in flight, is faster.
+      if (plan_shared(g, allow_compact, p) && p->threads >= 48) return PE_OK;
       Plan w, gl;
       const bool has_w = plan_warp(g, K, flags, allow_compact, &w);
       const bool has_g = plan_global(g, K, flags, allow_compact, &gl);

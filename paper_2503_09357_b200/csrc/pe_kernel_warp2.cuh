@@ -5,15 +5,20 @@
 // block still fits on chip when a whole warp shares it.  Inside a window the only things an
 // operator can wait for are (a) a predecessor that sits in the same window and (b) the
 // previous operator of its machine in the same window (Eqs. 7-8); both sit at lower lanes
-// because the order is topological.  The window is therefore resolved in rounds:
-//   set-up   each lane marks its operator "in this window, lane l" in the state, then reads
-//            its incoming edges once: a source that is already scheduled contributes its end
-//            time plus the cross-machine delay (Eqs. 11-13) at once; a source at a lower lane
-//            of the window is remembered (operator id and delay) and its lane joins `need`,
-//            as does the lane of the machine's previous operator (Eqs. 7-8);
-//   rounds   a lane whose `need` lanes have all finished takes the maximum of what it has and
-//            the remembered sources' end times plus delays, ends D^o later (Eq. 3), publishes;
-// the lowest unfinished lane is always ready, so the rounds end after at most 32 steps.
+// because the order is topological.  The window is therefore resolved in two steps.
+// Set-up: each lane marks its operator "in this window, lane l" in the state, then reads its
+// incoming edges once; a source that is already scheduled contributes its end time plus the
+// cross-machine delay (Eqs. 11-13) at once, a source at a lower lane of the window is
+// remembered, as is the machine's previous operator inside the window (Eqs. 7-8).  Then
+//   REG_SLOTS (no operator has more than three incoming edges): the remembered sources are
+//     (lane, delay) pairs in registers and the window is relaxed with shuffles: every lane
+//     repeatedly takes the maximum of what it has and its sources' current end times plus
+//     delays and ends D^o later (Eq. 3); the values rise to the window's longest-path solution
+//     and the loop stops when nothing changes - mostly long before the window's depth;
+//   otherwise: the remembered sources are operator ids (the inline ones) or the edge list
+//     itself, the lanes waited for form a mask `need`, and the window is resolved in rounds: a
+//     lane whose `need` lanes have finished evaluates once, from the state in shared memory, and
+//     publishes; the lowest unfinished lane is always ready, so at most 32 rounds.
 // Memory levels (Eqs. 16-19) do not depend on times: they are prefix sums along each
 // machine's lanes, formed once per window with shuffles.
 //
@@ -39,11 +44,13 @@ constexpr int kSlab = 128;
 
 // FLAT: one link class and no operator with more than three incoming edges: the three inline slots are
 // all there is, so the edge-list loops (and the `more` path) drop out of the window code.
-template <typename IdxT, bool BY_POS, int CLS, bool GRAPH_SMEM, bool TIMES, bool SLAB, bool FLAT>
+// REG_SLOTS: no operator has more than three incoming edges (whatever the link classes): in-window
+// dependences are kept as (lane, delay) in registers and resolved by shuffles.
+template <typename IdxT, bool BY_POS, int CLS, bool GRAPH_SMEM, bool TIMES, bool SLAB, bool FLAT, bool REG_SLOTS>
 __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, const uint8_t* __restrict__ nblob, int64_t K,
                                                              const uint8_t* __restrict__ assign,
                                                              const uint16_t* __restrict__ order, pe_outputs out,
-                                                             uint32_t flags, int* err, int warp_words) {
+                                                             uint32_t flags, int* err, int warp_words, int final_rounds) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   constexpr uint32_t FULL = 0xFFFFFFFFu;
   constexpr bool TWO_CLASS = CLS == 2;
@@ -126,7 +133,7 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
     const uint32_t below = same_dev & lt_mask;
     const int prev = below ? 31 - __clz(below) : -1;
     const bool last_on_dev = (same_dev >> lane) == 1u;
-    const uint32_t i_prev = __shfl_sync(FULL, i, prev < 0 ? lane : prev);
+    const uint32_t i_prev = REG_SLOTS ? 0u : __shfl_sync(FULL, i, prev < 0 ? lane : prev);
 
     // memory level along the machine's lanes (Eqs. 17-19): level before the window + prefix sum of A
     int32_t lv = dA;
@@ -147,97 +154,204 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
     __syncwarp();
     if (act && last_on_dev) lvl[j] = lv;
 
-    // Classify the incoming edges once.  A source that is already scheduled contributes its end
-    // time (+ delay) to r_base right away; a source that sits at a lower lane of this window becomes
-    // a "slot" (operator id | delay << 16) to be read when that lane has finished, and its lane joins
-    // `need`.  Edges beyond the inline ones that are in-window set `more`: they are re-read from the
-    // edge list at evaluation time.
-    uint32_t need = 0;
-    int32_t r_base = 0;
-    bool more = false;
-    const uint32_t none = (uint32_t)V;  // the sentinel: always "ended at 0"
-    uint32_t slot0 = none, slot1 = none, slot2 = none, slot_prev = none;
-    auto delay_of = [&](uint32_t lo, uint32_t hi, uint32_t w) -> uint32_t {
-      const uint32_t xp = w & 0xFFu;
-      uint32_t delay = lo >> 16;
-      if (NEED_CLS) {
-        const uint32_t cl = gp.cls[xp * D + j];
-        if (TWO_CLASS) delay = cl == 1u ? hi : delay;
-        if (cl == 0xFFu) {
-          delay = 0;
-          if ((lo & 0xFFFFu) != none && xp != j) st |= PE_STATUS_NO_CHANNEL;
-        }
-      }
-      return xp != j ? delay : 0u;
-    };
-    auto classify = [&](uint32_t lo, uint32_t hi, uint32_t& slot, bool inline_slot) {
-      const uint32_t p = lo & 0xFFFFu;
-      const uint32_t w = state[p];
-      const uint32_t dly = delay_of(lo, hi, w);
-      if (w < kDoneLimit) {
-        r_base = max(r_base, (int32_t)((w >> 8) + dly));
-      } else {
-        const uint32_t l = (w >> 8) & 31u;
-        if (w < kInWindowEnd && l < (uint32_t)lane) {
-          need |= 1u << l;
-          if (inline_slot) slot = p | (dly << 16);
-          else more = true;
-        } else {
-          st |= PE_STATUS_ORDER_INVALID;  // a predecessor that is not before this operator
-        }
-      }
-    };
-    if (act) {
-      uint32_t unused = none;
-      classify(rec.z, rec.w, slot0, true);
-      if (TWO_CLASS) {
-        const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
-        for (int q = 1; q < indeg; ++q) classify(ed[q].x, ed[q].y, unused, false);
-      } else {
-        classify(rec.w, 0u, slot1, true);
-        classify(third, 0u, slot2, true);
-        if (!FLAT && indeg > 3) {
-          const uint32_t* ed = gp.edges + rec.x;
-          for (int q = 2; q < indeg; ++q) classify(ed[q], 0u, unused, false);
-        }
-      }
-      if (prev < 0) {
-        r_base = max(r_base, free_at[j]);
-      } else {
-        need |= 1u << prev;  // Eqs. 7-8: after the machine's previous operator
-        slot_prev = i_prev;
-      }
-    }
-
-    // rounds: the lowest unfinished lane never waits, so every round finishes at least one
-    auto slot_time = [&](uint32_t sl) -> int32_t { return (int32_t)((state[sl & 0xFFFFu] >> 8) + (sl >> 16)); };
-    bool pend = act;
     int32_t s = 0, e = 0;
-    uint32_t pendmask;
-    while ((pendmask = __ballot_sync(FULL, pend)) != 0) {
-      if (pend && (need & pendmask) == 0) {
-        int32_t v = max(max(r_base, slot_time(slot0)), max(slot_time(slot1), max(slot_time(slot2), slot_time(slot_prev))));
-        if (!FLAT && more) {  // in-window sources among the edges kept in the edge list: all finished by now
-          if (TWO_CLASS) {
-            const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
-            for (int q = 1; q < indeg; ++q) {
-              const uint32_t w = state[ed[q].x & 0xFFFFu];
-              v = max(v, (int32_t)((w >> 8) + delay_of(ed[q].x, ed[q].y, w)));
-            }
-          } else {
-            const uint32_t* ed = gp.edges + rec.x;
-            for (int q = 2; q < indeg; ++q) {
-              const uint32_t w = state[ed[q] & 0xFFFFu];
-              v = max(v, (int32_t)((w >> 8) + delay_of(ed[q], 0u, w)));
-            }
+    if constexpr (REG_SLOTS) {
+      // Classify the incoming edges once.  A source that is already scheduled contributes its end
+      // time (+ delay) to r_base right away.  A source that sits at a lower lane of this window becomes
+      // a "slot": the lane it sits at and the delay that applies (Eqs. 11-13; the machines of both ends
+      // are known by now).  With at most three incoming edges per operator three slots suffice.  The
+      // previous operator of the machine inside the window (Eqs. 7-8) is a fourth slot with delay 0.
+      constexpr int32_t kNever = -(1 << 29);   // delay of an empty slot: never wins the maximum
+      int32_t r_base = 0;
+      int nslots = 0;
+      uint32_t depmask = 0;   // lanes of this window this operator waits for
+      int l0 = lane, l1 = lane, l2 = lane;
+      int32_t d0 = kNever, d1 = kNever, d2 = kNever;
+      const uint32_t none = (uint32_t)V;  // the sentinel: always "ended at 0"
+      auto delay_of = [&](uint32_t lo, uint32_t hi, uint32_t w) -> uint32_t {
+        const uint32_t xp = w & 0xFFu;
+        uint32_t delay = lo >> 16;
+        if (NEED_CLS) {
+          const uint32_t cl = gp.cls[xp * D + j];
+          if (TWO_CLASS) delay = cl == 1u ? hi : delay;
+          if (cl == 0xFFu) {
+            delay = 0;
+            if ((lo & 0xFFFFu) != none && xp != j) st |= PE_STATUS_NO_CHANNEL;
           }
         }
-        s = v;
-        e = s + dur;
-        state[i] = ((uint32_t)e << 8) | j;
-        pend = false;
+        return xp != j ? delay : 0u;
+      };
+      auto classify = [&](uint32_t lo, uint32_t hi) {
+        const uint32_t p = lo & 0xFFFFu;
+        const uint32_t w = state[p];
+        const uint32_t dly = delay_of(lo, hi, w);
+        if (w < kDoneLimit) {
+          r_base = max(r_base, (int32_t)((w >> 8) + dly));
+        } else {
+          const uint32_t l = (w >> 8) & 31u;
+          if (w < kInWindowEnd && l < (uint32_t)lane) {
+            if (nslots == 0) { l0 = (int)l; d0 = (int32_t)dly; }
+            else if (nslots == 1) { l1 = (int)l; d1 = (int32_t)dly; }
+            else if (nslots == 2) { l2 = (int)l; d2 = (int32_t)dly; }
+            ++nslots;
+            depmask |= 1u << l;
+          } else {
+            st |= PE_STATUS_ORDER_INVALID;  // a predecessor that is not before this operator
+          }
+        }
+      };
+      int lp = lane;
+      int32_t dp = kNever;
+      if (act) {
+        classify(rec.z, rec.w);
+        if (TWO_CLASS) {
+          const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
+          for (int q = 1; q < indeg; ++q) classify(ed[q].x, ed[q].y);
+        } else {
+          classify(rec.w, 0u);
+          classify(third, 0u);
+          if (!FLAT && indeg > 3) {
+            const uint32_t* ed = gp.edges + rec.x;
+            for (int q = 2; q < indeg; ++q) classify(ed[q], 0u);
+          }
+        }
+        if (prev < 0) r_base = max(r_base, free_at[j]);
+        else { lp = prev; dp = 0; depmask |= 1u << prev; }   // Eqs. 7-8: after the machine's previous operator
       }
-      __syncwarp();
+
+      // Two ways to resolve the window, both exchanging end times by shuffles only.
+      // Relaxation (many warps per SM, instruction issue is what limits): every lane starts from what
+      // it knows (r_base) and repeatedly takes the maximum over its slots of the slot lane's current
+      // end time plus delay; all dependences point to lower lanes, so the values rise monotonically
+      // to the window's longest-path solution and the loop stops when nothing changes - usually long
+      // before the window's depth, because most dependences do not bind.
+      // Rounds (few warps per SM, latency is what limits): a lane evaluates once, when every lane it
+      // depends on is final; exactly (depth of the window) rounds, but the loop-carried chain is a
+      // ballot and a mask test instead of shuffle, maximum, compare and vote.
+      e = r_base + dur;
+      if (!final_rounds) {
+        if (__any_sync(FULL, depmask != 0)) {
+          for (int it = 0; it < 34; ++it) {
+            int32_t v = r_base;
+            v = max(v, __shfl_sync(FULL, e, l0) + d0);
+            v = max(v, __shfl_sync(FULL, e, l1) + d1);
+            v = max(v, __shfl_sync(FULL, e, l2) + d2);
+            v = max(v, __shfl_sync(FULL, e, lp) + dp);
+            const int32_t en = v + dur;
+            const bool changed = en != e;
+            e = en;
+            if (!__any_sync(FULL, changed)) break;
+          }
+        }
+      } else {
+        bool fin = depmask == 0;
+        for (int it = 0; it < 33; ++it) {
+          const uint32_t fm = __ballot_sync(FULL, fin);
+          if (fm == FULL) break;
+          int32_t v = r_base;
+          v = max(v, __shfl_sync(FULL, e, l0) + d0);
+          v = max(v, __shfl_sync(FULL, e, l1) + d1);
+          v = max(v, __shfl_sync(FULL, e, l2) + d2);
+          v = max(v, __shfl_sync(FULL, e, lp) + dp);
+          if (!fin && (depmask & ~fm) == 0) { e = v + dur; fin = true; }
+        }
+      }
+      s = e - dur;
+      if (act) state[i] = ((uint32_t)e << 8) | j;
+
+    } else {
+      // Classify the incoming edges once.  A source that is already scheduled contributes its end
+      // time (+ delay) to r_base right away; a source that sits at a lower lane of this window becomes
+      // a "slot" (operator id | delay << 16) to be read when that lane has finished, and its lane joins
+      // `need`.  Edges beyond the inline ones that are in-window set `more`: they are re-read from the
+      // edge list at evaluation time.
+      uint32_t need = 0;
+      int32_t r_base = 0;
+      bool more = false;
+      const uint32_t none = (uint32_t)V;  // the sentinel: always "ended at 0"
+      uint32_t slot0 = none, slot1 = none, slot2 = none, slot_prev = none;
+      auto delay_of = [&](uint32_t lo, uint32_t hi, uint32_t w) -> uint32_t {
+        const uint32_t xp = w & 0xFFu;
+        uint32_t delay = lo >> 16;
+        if (NEED_CLS) {
+          const uint32_t cl = gp.cls[xp * D + j];
+          if (TWO_CLASS) delay = cl == 1u ? hi : delay;
+          if (cl == 0xFFu) {
+            delay = 0;
+            if ((lo & 0xFFFFu) != none && xp != j) st |= PE_STATUS_NO_CHANNEL;
+          }
+        }
+        return xp != j ? delay : 0u;
+      };
+      auto classify = [&](uint32_t lo, uint32_t hi, uint32_t& slot, bool inline_slot) {
+        const uint32_t p = lo & 0xFFFFu;
+        const uint32_t w = state[p];
+        const uint32_t dly = delay_of(lo, hi, w);
+        if (w < kDoneLimit) {
+          r_base = max(r_base, (int32_t)((w >> 8) + dly));
+        } else {
+          const uint32_t l = (w >> 8) & 31u;
+          if (w < kInWindowEnd && l < (uint32_t)lane) {
+            need |= 1u << l;
+            if (inline_slot) slot = p | (dly << 16);
+            else more = true;
+          } else {
+            st |= PE_STATUS_ORDER_INVALID;  // a predecessor that is not before this operator
+          }
+        }
+      };
+      if (act) {
+        uint32_t unused = none;
+        classify(rec.z, rec.w, slot0, true);
+        if (TWO_CLASS) {
+          const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
+          for (int q = 1; q < indeg; ++q) classify(ed[q].x, ed[q].y, unused, false);
+        } else {
+          classify(rec.w, 0u, slot1, true);
+          classify(third, 0u, slot2, true);
+          if (!FLAT && indeg > 3) {
+            const uint32_t* ed = gp.edges + rec.x;
+            for (int q = 2; q < indeg; ++q) classify(ed[q], 0u, unused, false);
+          }
+        }
+        if (prev < 0) {
+          r_base = max(r_base, free_at[j]);
+        } else {
+          need |= 1u << prev;  // Eqs. 7-8: after the machine's previous operator
+          slot_prev = i_prev;
+        }
+      }
+
+      // rounds: the lowest unfinished lane never waits, so every round finishes at least one
+      auto slot_time = [&](uint32_t sl) -> int32_t { return (int32_t)((state[sl & 0xFFFFu] >> 8) + (sl >> 16)); };
+      bool pend = act;
+      uint32_t pendmask;
+      while ((pendmask = __ballot_sync(FULL, pend)) != 0) {
+        if (pend && (need & pendmask) == 0) {
+          int32_t v = max(max(r_base, slot_time(slot0)), max(slot_time(slot1), max(slot_time(slot2), slot_time(slot_prev))));
+          if (!FLAT && more) {  // in-window sources among the edges kept in the edge list: all finished by now
+            if (TWO_CLASS) {
+              const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
+              for (int q = 1; q < indeg; ++q) {
+                const uint32_t w = state[ed[q].x & 0xFFFFu];
+                v = max(v, (int32_t)((w >> 8) + delay_of(ed[q].x, ed[q].y, w)));
+              }
+            } else {
+              const uint32_t* ed = gp.edges + rec.x;
+              for (int q = 2; q < indeg; ++q) {
+                const uint32_t w = state[ed[q] & 0xFFFFu];
+                v = max(v, (int32_t)((w >> 8) + delay_of(ed[q], 0u, w)));
+              }
+            }
+          }
+          s = v;
+          e = s + dur;
+          state[i] = ((uint32_t)e << 8) | j;
+          pend = false;
+        }
+        __syncwarp();
+      }
+
     }
 
     if (act && last_on_dev) free_at[j] = e;

@@ -9,24 +9,29 @@ static int launch4(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* a
                    uint32_t flags, const pe_outputs& out, unsigned grid, cudaStream_t stream) {
   auto go = [&](auto kern) -> int {
     if (!set_smem(kern, p.smem)) return PE_ERR_CUDA;
+    // few warps per SM: the window loop with the shorter loop-carried chain (see the kernel)
+    const int final_rounds = p.threads / 32 < 8 ? 1 : 0;
     kern<<<grid, p.threads, p.smem, stream>>>(g->nview, g->d_nblob, K, assign, order, out, flags, g->d_error,
-                                               p.warp_words);
+                                               p.warp_words, final_rounds);
     return PE_OK;
   };
   constexpr bool kCanFlat = CLS == 0;
-  const bool flat = kCanFlat && g->max_indeg <= 3;
+  const bool reg = g->max_indeg <= 3;   // in-window dependences fit the register slots
+  const bool flat = kCanFlat && reg;
+#define PE_W2(SLAB, FLAT, REG)                                                                       \
+  return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, SLAB, FLAT, REG>)  \
+                   : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, SLAB, FLAT, REG>)
   if (flat) {
-    if (p.slab)
-      return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, true, kCanFlat>)
-                       : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, true, kCanFlat>);
-    return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, false, kCanFlat>)
-                     : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, false, kCanFlat>);
+    if (p.slab) PE_W2(true, kCanFlat, true);
+    PE_W2(false, kCanFlat, true);
   }
-  if (p.slab)
-    return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, true, false>)
-                     : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, true, false>);
-  return out.start ? go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, true, false, false>)
-                   : go(pe_eval_warp2_kernel<IdxT, BY_POS, CLS, GRAPH_SMEM, false, false, false>);
+  if (reg) {
+    if (p.slab) PE_W2(true, false, true);
+    PE_W2(false, false, true);
+  }
+  if (p.slab) PE_W2(true, false, false);
+  PE_W2(false, false, false);
+#undef PE_W2
 }
 
 template <bool BY_POS>
