@@ -35,6 +35,11 @@
 // The paper's own DualPipe bubble figures for PP = 4 and 8 (Section V-A) are "parity
 // unpinned": the schedule behind them and its microbatch count are not printed.
 //
+// The second function of this file, pe_oracle_decode (at the end), states the step before
+// evaluation - turning an arbitrary priority list into a priority order - and is pinned by
+// tests/test_decode_pins.py: brute force over all topological orders of tiny DAGs, the
+// edge-free and chain cases, idempotence, and the input generator's own random-key sort.
+//
 // Arrays are candidate-interleaved: element (row, c) of a [R][K] array is at row*K + c.
 #include <cstdint>
 #include <vector>
@@ -164,6 +169,69 @@ extern "C" int pe_oracle_eval(int32_t V, int32_t E, const int32_t* edge_src, con
       if (peak_mem) peak_mem[(size_t)j * (size_t)K + (size_t)c] = peak[j];
     }
     if (status) status[c] = st;
+  }
+  return 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Priority-list decoding: the step before evaluation.  TEST INFRASTRUCTURE ONLY, like the rest.
+//
+// Section IV frames heuristics for this problem as "priority dispatch rule-based algorithms".
+// The rule written out here: a candidate gives every operation a priority rank through a list
+// (list[r] = the operation of rank r, rank 0 the most urgent; any permutation of I, it need not
+// respect the precedence edges B), and the priority order pi is built one position at a time:
+// among the operations not yet placed whose predecessors in B have all been placed, the one of
+// smallest rank comes next.  pi is therefore a topological order of G_m, which is what the
+// evaluation above asks for, and a list that already is one is returned unchanged.
+//
+// A list that is not a permutation (an entry >= V, an operation twice) sets kStatusOrderInvalid
+// and leaves that candidate's order unspecified.
+// Arrays are candidate-interleaved like everything else: element (row, c) at row*K + c.
+#include <queue>
+
+extern "C" int pe_oracle_decode(int32_t V, int32_t E, const int32_t* edge_src, const int32_t* edge_dst, int64_t K,
+                                int64_t c_begin, int64_t c_end, const void* list, int order_bytes, void* order,
+                                uint32_t* status) {
+  if (V <= 0 || E < 0 || K < 0 || c_begin < 0 || c_end > K || !list || !order) return -1;
+  if (order_bytes != 2 && order_bytes != 4) return -1;
+  for (int32_t b = 0; b < E; ++b)
+    if (edge_src[b] < 0 || edge_src[b] >= V || edge_dst[b] < 0 || edge_dst[b] >= V) return -1;
+  auto get = [&](const void* a, size_t at) -> uint32_t {
+    return order_bytes == 2 ? (uint32_t)((const uint16_t*)a)[at] : ((const uint32_t*)a)[at];
+  };
+  auto put = [&](size_t at, uint32_t v) {
+    if (order_bytes == 2) ((uint16_t*)order)[at] = (uint16_t)v;
+    else ((uint32_t*)order)[at] = v;
+  };
+  std::vector<std::vector<int32_t>> succ(V);
+  std::vector<int32_t> indeg(V, 0);
+  for (int32_t b = 0; b < E; ++b) { succ[edge_src[b]].push_back(edge_dst[b]); indeg[edge_dst[b]]++; }
+  std::vector<int64_t> rank(V);
+  std::vector<int32_t> waiting(V);
+  for (int64_t c = c_begin; c < c_end; ++c) {
+    bool ok = true;
+    for (int32_t i = 0; i < V; ++i) rank[i] = -1;
+    for (int32_t r = 0; r < V; ++r) {
+      const uint32_t i = get(list, (size_t)r * (size_t)K + (size_t)c);
+      if (i >= (uint32_t)V || rank[i] >= 0) { ok = false; continue; }
+      rank[i] = r;
+    }
+    if (status) status[c] = ok ? 0u : kStatusOrderInvalid;
+    if (!ok) continue;
+    // ranks of the operations that may come next; the smallest is on top
+    std::priority_queue<int64_t, std::vector<int64_t>, std::greater<int64_t>> ready;
+    for (int32_t i = 0; i < V; ++i) { waiting[i] = indeg[i]; if (indeg[i] == 0) ready.push(rank[i]); }
+    int32_t k = 0;
+    while (!ready.empty()) {
+      const int64_t r = ready.top();
+      ready.pop();
+      const uint32_t i = get(list, (size_t)r * (size_t)K + (size_t)c);
+      put((size_t)k * (size_t)K + (size_t)c, i);
+      ++k;
+      for (int32_t s : succ[i])
+        if (--waiting[s] == 0) ready.push(rank[s]);
+    }
+    if (k != V) return -2;  // the edge list has a cycle
   }
   return 0;
 }

@@ -41,6 +41,9 @@ def _load():
         lib.pe_oracle_eval.argtypes = [ctypes.c_int32, ctypes.c_int32, P, P, P, P, P, ctypes.c_int32, ctypes.c_int32,
                                        P, P, P, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, P, P, ctypes.c_int,
                                        ctypes.c_uint32, P, P, P, P, P, P]
+        lib.pe_oracle_decode.restype = ctypes.c_int
+        lib.pe_oracle_decode.argtypes = [ctypes.c_int32, ctypes.c_int32, P, P, ctypes.c_int64, ctypes.c_int64,
+                                         ctypes.c_int64, P, ctypes.c_int, P, P]
         _lib = lib
     return _lib
 
@@ -108,3 +111,31 @@ def select_best(makespan, status, reject_mask=0xFFFFFFFF):
         if best_c < 0 or int(makespan[c]) < best:
             best, best_c = int(makespan[c]), c
     return best_c, best, count
+
+
+def decode(w, plist, threads=1):
+    """Priority-list decoding (see pe_oracle.cpp): plist is u16/u32 [V, K], plist[r, c] = the operation of
+    rank r of candidate c.  Returns (order [V, K] of the same dtype, status [K] uint32)."""
+    V = int(w.num_ops)
+    plist = np.ascontiguousarray(plist)
+    assert plist.dtype in (np.uint16, np.uint32) and plist.shape[0] == V
+    K = plist.shape[1]
+    src, dst = _c(w.edge_src, np.int32), _c(w.edge_dst, np.int32)
+    order = np.zeros_like(plist)
+    status = np.zeros(K, np.uint32)
+    lib = _load()
+
+    def run(lo, hi):
+        rc = lib.pe_oracle_decode(V, int(src.shape[0]), _p(src), _p(dst), K, lo, hi, _p(plist), plist.dtype.itemsize,
+                                  _p(order), _p(status))
+        if rc != 0:
+            raise RuntimeError(f"pe_oracle_decode failed with code {rc}")
+
+    threads = max(1, min(int(threads), K)) if K > 0 else 1
+    if threads == 1:
+        run(0, K)
+    else:
+        cuts = [K * t // threads for t in range(threads + 1)]
+        with ThreadPoolExecutor(threads) as pool:
+            list(pool.map(lambda t: run(cuts[t], cuts[t + 1]), range(threads)))
+    return order, status
