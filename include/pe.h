@@ -173,6 +173,26 @@ int pe_eval_batch_host(pe_graph* g, int64_t K, const uint8_t* host_assign, const
 int pe_eval_batch_noalloc(pe_graph* g, int64_t K, const uint8_t* assign, const void* order, int order_bytes,
                           uint32_t flags, const pe_outputs* out, void* cuda_stream);
 
+/* Priority-list decoding: the step in front of pe_eval_batch (Section IV: heuristics for this problem are
+ * "priority dispatch rule-based algorithms"; Eq. 8 needs the resulting order to be consistent with B).
+ * A candidate ranks the operators through a list; the priority order is then built position by position:
+ * among the operators not yet placed whose predecessors in B have all been placed, the one of smallest rank
+ * comes next.  The result is a topological order of G_m - a valid `order` argument of pe_eval_batch - and a
+ * list that already is one comes back unchanged.
+ *   list        device, uint16_t [V*K]: list_c[r] = operator of rank r (0 = most urgent) at r*K + c; any
+ *               permutation of the operators, it need not respect the edges
+ *   order_bytes 2 (uint16_t entries); 4 is PE_ERR_UNSUPPORTED, as are V > 65536 and in-degrees above 255
+ *   flags       0, or PE_VARIANT_SHARED / PE_VARIANT_GLOBAL to force where the per-candidate state lives
+ *   order       device, uint16_t [V*K], out: pi_c[k] at k*K + c
+ *   status      device, [K], out, may be NULL: PE_STATUS_ORDER_INVALID where the list is not a permutation
+ *               (an entry >= V or an operator twice); that candidate's order is then left unwritten
+ *   workspace   device scratch of at least pe_decode_workspace_bytes() bytes (may be 0), 256-byte aligned
+ * Asynchronous on `cuda_stream`; never synchronises.  K = 0 is a successful no-op. */
+size_t pe_decode_workspace_bytes(const pe_graph* g, int64_t K, uint32_t flags);
+int pe_decode_variant(const pe_graph* g, int64_t K, uint32_t flags); /* PE_VARIANT_SHARED or _GLOBAL; negative = error */
+int pe_decode_priority(pe_graph* g, int64_t K, const void* list, int order_bytes, uint32_t flags, void* order,
+                       uint32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Selection step after an evaluation (Eq. 1: the objective is the makespan; Section III: only
  * arrangements within every machine's memory limit are valid): among K evaluated candidates find the
  * one with the smallest makespan whose status has none of the bits in `reject_mask` set

@@ -63,6 +63,12 @@ _lib.pe_eval_batch_host.argtypes = [_P, ctypes.c_int64, _P, _P, ctypes.c_int, ct
 _lib.pe_eval_batch_noalloc.restype = ctypes.c_int
 _lib.pe_eval_batch_noalloc.argtypes = [_P, ctypes.c_int64, _P, _P, ctypes.c_int, ctypes.c_uint32,
                                        ctypes.POINTER(pe_outputs), _P]
+_lib.pe_decode_workspace_bytes.restype = ctypes.c_size_t
+_lib.pe_decode_workspace_bytes.argtypes = [_P, ctypes.c_int64, ctypes.c_uint32]
+_lib.pe_decode_variant.restype = ctypes.c_int
+_lib.pe_decode_variant.argtypes = [_P, ctypes.c_int64, ctypes.c_uint32]
+_lib.pe_decode_priority.restype = ctypes.c_int
+_lib.pe_decode_priority.argtypes = [_P, ctypes.c_int64, _P, ctypes.c_int, ctypes.c_uint32, _P, _P, _P, ctypes.c_size_t, _P]
 _lib.pe_select_best.restype = ctypes.c_int
 _lib.pe_select_best.argtypes = [ctypes.c_int64, _P, _P, ctypes.c_uint32, _P, _P]
 _lib.pe_graph_poll_error.restype = ctypes.c_int
@@ -175,6 +181,21 @@ def pe_select_best(K, makespan_ptr, status_ptr, reject_mask, result_ptr, stream=
                                result_ptr, stream or None)
 
 
+def pe_decode_workspace_bytes(handle, K: int, flags: int = 0) -> int:
+    return int(_lib.pe_decode_workspace_bytes(handle, int(K), int(flags)))
+
+
+def pe_decode_variant(handle, K: int, flags: int = 0) -> int:
+    return int(_lib.pe_decode_variant(handle, int(K), int(flags)))
+
+
+def pe_decode_priority(handle, K, list_ptr, order_bytes, flags, order_ptr, status_ptr=0, workspace=0, workspace_bytes=0,
+                       stream=0) -> int:
+    """Raw call: priority lists -> topological priority orders (device pointers)."""
+    return _lib.pe_decode_priority(handle, int(K), list_ptr or None, int(order_bytes), int(flags), order_ptr or None,
+                                   status_ptr or None, workspace or None, int(workspace_bytes), stream or None)
+
+
 def pe_graph_poll_error(handle, stream=0) -> int:
     return _lib.pe_graph_poll_error(handle, stream or None)
 
@@ -237,6 +258,25 @@ class Graph:
             raise PeError(rc, "pe_select_best")
         idx, mk, cnt, _ = res.tolist()
         return idx, mk, cnt
+
+    def decode_priority(self, plist, flags=0, stream=None):
+        """plist: cuda int16 [V, K] holding u16 operator ids, plist[r, c] = operator of rank r of candidate c.
+        Returns (order, status): the topological priority orders (same shape and dtype) and a uint32-bit
+        status per candidate (int32 tensor).  Asynchronous on `stream` (default: torch's current stream)."""
+        import torch
+        K = int(plist.shape[1])
+        assert plist.is_cuda and plist.is_contiguous() and tuple(plist.shape) == (self.V, K) and plist.element_size() == 2
+        dev = torch.device("cuda", self.device)
+        order = torch.empty_like(plist)
+        status = torch.empty(K, dtype=torch.int32, device=dev)
+        n = pe_decode_workspace_bytes(self.handle, K, flags)
+        ws = torch.empty(max(n, 256), dtype=torch.uint8, device=dev)
+        s = torch.cuda.current_stream(self.device).cuda_stream if stream is None else stream
+        rc = pe_decode_priority(self.handle, K, plist.data_ptr(), 2, flags, order.data_ptr(), status.data_ptr(),
+                                ws.data_ptr(), n, s)
+        if rc != PE_OK:
+            raise PeError(rc, "pe_decode_priority")
+        return order, status
 
     def eval_batch(self, assign, order, flags=0, out=None, workspace=None, want_times=True, stream=None):
         """assign: cuda uint8 [V, K]; order: cuda int16/int32 [V, K] holding u16/u32 bits.

@@ -429,7 +429,10 @@ extern "C" int pe_eval_variant(const pe_graph* g, int64_t K, uint32_t flags) {
   return rc != PE_OK ? rc : p.variant;
 }
 
-extern "C" int64_t pe_kernel_launches(void) { return pe::g_launches.load(std::memory_order_relaxed); }
+namespace pe { extern std::atomic<int64_t> g_decode_launches; }
+extern "C" int64_t pe_kernel_launches(void) {
+  return pe::g_launches.load(std::memory_order_relaxed) + pe::g_decode_launches.load(std::memory_order_relaxed);
+}
 
 extern "C" int pe_eval_batch(pe_graph* g, int64_t K, const uint8_t* assign, const void* order, int order_bytes,
                              uint32_t flags, const pe_outputs* out, void* workspace, size_t workspace_bytes,

@@ -190,6 +190,29 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
     std::memcpy(nblob.data() + nv.cap, cap, (size_t)D * 4);
   }
 
+  // forward view (successor lists) for priority-list decoding
+  std::vector<uint8_t> fblob;
+  g->fwd_ok = V <= 65536 && mdeg <= 255;
+  g->d_fwd = nullptr;
+  std::memset(&g->fview, 0, sizeof(g->fview));
+  if (g->fwd_ok) {
+    PeFwdView& fv = g->fview;
+    fv.V = V; fv.E = E;
+    uint64_t fat = 0;
+    fv.ptr = (uint32_t)fat;   fat = align16(fat + (uint64_t)(V + 1) * 4);
+    fv.succ = (uint32_t)fat;  fat = align16(fat + (uint64_t)E * 2);
+    fv.indeg = (uint32_t)fat; fat = align16(fat + (uint64_t)V);
+    fv.bytes = (uint32_t)fat;
+    fblob.assign(fv.bytes, 0);
+    uint32_t* fptr = (uint32_t*)(fblob.data() + fv.ptr);
+    uint16_t* fsucc = (uint16_t*)(fblob.data() + fv.succ);
+    uint8_t* findeg = fblob.data() + fv.indeg;
+    for (int32_t b = 0; b < E; ++b) fptr[d->edge_src[b] + 1]++;
+    for (int32_t i = 0; i < V; ++i) { fptr[i + 1] += fptr[i]; findeg[i] = (uint8_t)ops[i].indeg; }
+    std::vector<uint32_t> ffill(fptr, fptr + V);
+    for (int32_t b = 0; b < E; ++b) fsucc[ffill[d->edge_src[b]]++] = (uint16_t)d->edge_dst[b];
+  }
+
   cudaDeviceProp prop;
   int prev = -1;
   bool ok = cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(cuda_device) == cudaSuccess &&
@@ -204,6 +227,9 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
     if (ok && narrow)
       ok = cudaMalloc((void**)&g->d_nblob, nblob.size()) == cudaSuccess &&
            cudaMemcpy(g->d_nblob, nblob.data(), nblob.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    if (ok && g->fwd_ok)
+      ok = cudaMalloc((void**)&g->d_fwd, fblob.size()) == cudaSuccess &&
+           cudaMemcpy(g->d_fwd, fblob.data(), fblob.size(), cudaMemcpyHostToDevice) == cudaSuccess;
     if (ok) {
       ok = cudaStreamCreateWithFlags(&g->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
            cudaStreamCreateWithFlags(&g->copy_out, cudaStreamNonBlocking) == cudaSuccess &&
@@ -220,6 +246,7 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
     if (g->d_blob) cudaFree(g->d_blob);
     if (g->d_error) cudaFree(g->d_error);
     if (g->d_nblob) cudaFree(g->d_nblob);
+    if (g->d_fwd) cudaFree(g->d_fwd);
     if (g->copy_in) cudaStreamDestroy(g->copy_in);
     if (g->copy_out) cudaStreamDestroy(g->copy_out);
     if (g->ev_begin) cudaEventDestroy(g->ev_begin);
@@ -248,6 +275,7 @@ extern "C" int pe_destroy(pe_graph* g) {
   for (int q = 0; q < pe_graph::kMaxChunks; ++q) { cudaEventDestroy(g->ev_in[q]); cudaEventDestroy(g->ev_done[q]); }
   bool ok = cudaFree(g->d_blob) == cudaSuccess && cudaFree(g->d_error) == cudaSuccess;
   if (g->d_nblob) ok = cudaFree(g->d_nblob) == cudaSuccess && ok;
+  if (g->d_fwd) ok = cudaFree(g->d_fwd) == cudaSuccess && ok;
   if (prev >= 0) cudaSetDevice(prev);
   delete g;
   return ok ? PE_OK : PE_ERR_CUDA;

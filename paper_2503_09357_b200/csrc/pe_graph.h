@@ -61,6 +61,16 @@ struct PeNarrowView {
   uint32_t bytes;     // total, multiple of 16
 };
 
+// Forward view of the DAG for priority-list decoding, built when V <= 65536 and no operator has
+// more than 255 incoming edges: successors of operator i are succ[ptr[i] .. ptr[i+1]).
+struct PeFwdView {
+  int32_t V, E;
+  uint32_t ptr;    // uint32[V + 1]
+  uint32_t succ;   // uint16[E]
+  uint32_t indeg;  // uint8[V]
+  uint32_t bytes;  // total, multiple of 16
+};
+
 struct pe_graph {
   int32_t V, E, D, L;
   int device;
@@ -73,6 +83,9 @@ struct pe_graph {
   bool narrow_ok;      // the compact encoding exists
   PeNarrowView nview;
   uint8_t* d_nblob;    // device copy of the compact encoding (nullptr if !narrow_ok)
+  bool fwd_ok;         // the forward view exists
+  PeFwdView fview;
+  uint8_t* d_fwd;      // device copy of the forward view (nullptr if !fwd_ok)
   int* d_error;        // device status word (0 = ok)
   // pe_eval_batch_host pipelines copies and kernels over candidate chunks: one stream per copy
   // direction and one event per chunk and stage, created with the graph; `host_mutex` serialises
