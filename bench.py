@@ -286,6 +286,7 @@ def run_ours(args):
     d2h = sum(v.numel() * v.element_size() for v in d_out.values())
 
     others = None
+    decode = []
     if rank == 0 and world == 1 and args.all_workloads:
         # free the headline's buffers, then time every other configuration (device-resident, fewer steps)
         del d_assign, d_order, d_out, ws, h_out, houts, outs
@@ -318,6 +319,36 @@ def run_ours(args):
                            "gbs": oalg / (ms * 1e-3) / 1e9})
             og.close()
             del da, do, oout, ows
+            torch.cuda.empty_cache()
+        # the step in front of the path: priority-list decoding, on uniformly random lists (device-made:
+        # argsort of random numbers per candidate), K * V = 2^28 per workload
+        decode = []
+        for name in sorted(WORKLOADS):
+            if name.endswith("_D64") or name == "tiny_pipeline":
+                continue                                  # decoding does not depend on the machines
+            ow = WORKLOADS[name]()
+            oV = ow.num_ops
+            oK = int(min(ow.num_candidates, max(1024, (1 << 28) // oV)))
+            og = pe.Graph(ow, device=local_rank)
+            gen = torch.Generator(device=dev); gen.manual_seed(oV)
+            plist = torch.argsort(torch.rand((oV, oK), device=dev, generator=gen), dim=0).to(torch.int16).contiguous()
+            for _ in range(2):
+                og.decode_priority(plist)
+            torch.cuda.synchronize(dev)
+            times = []
+            for _ in range(5):
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream); dorder, dstatus = og.decode_priority(plist); e1.record(stream)
+                torch.cuda.synchronize(dev)
+                times.append(e0.elapsed_time(e1))
+            ms = statistics.mean(times)
+            assert int(dstatus.abs().max()) == 0
+            dalg = oK * oV * 4 + oK * 4                    # list in, order out, status
+            decode.append({"workload": name, "V": oV, "K": oK,
+                           "kernel_variant": pe.VARIANT_NAMES[pe.pe_decode_variant(og.handle, oK, 0)], "ms": ms,
+                           "op_decodes_per_s": oK * oV / (ms * 1e-3), "gbs": dalg / (ms * 1e-3) / 1e9})
+            og.close()
+            del plist, dorder, dstatus
             torch.cuda.empty_cache()
 
     if rank == 0:
@@ -359,6 +390,9 @@ def run_ours(args):
             for o in others:
                 o["frac"] = o["gbs"] / peak
             line["other_workloads"] = others
+            for o in decode:
+                o["frac"] = o["gbs"] / peak
+            line["decode"] = decode
         print(json.dumps(line), flush=True)
     g.close()
     if world > 1:

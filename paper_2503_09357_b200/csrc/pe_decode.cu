@@ -83,9 +83,13 @@ __global__ void __launch_bounds__(256) pe_decode_kernel(PeFwdView f, const uint8
   uint64_t L2 = 0;
 
   auto add = [&](uint32_t r) {   // rank r becomes available
-    L0[(r >> 5) * pitch] |= 1u << (r & 31u);
-    L1[(r >> 10) * pitch] |= 1u << ((r >> 5) & 31u);
-    L2 |= 1ull << (r >> 10);
+    uint32_t* p0 = L0 + (r >> 5) * pitch;
+    const uint32_t w0 = *p0;
+    *p0 = w0 | (1u << (r & 31u));
+    if (w0 == 0u) {              // the word was empty: the levels above learn of it
+      L1[(r >> 10) * pitch] |= 1u << ((r >> 5) & 31u);
+      L2 |= 1ull << (r >> 10);
+    }
   };
 
   for (int i = 0; i < V; ++i) word[(uint32_t)i * pitch] = (uint32_t)fp.indeg[i] << 16;
@@ -110,10 +114,7 @@ __global__ void __launch_bounds__(256) pe_decode_kernel(PeFwdView f, const uint8
         const int r = r0 + u;
         if (r < V) {
           const uint32_t i = cur[u];
-          if (STATE_SMEM) {
-            uint32_t* pair = lst + (uint32_t)(r >> 1) * pitch;
-            *pair = (r & 1) ? ((*pair & 0xFFFFu) | (i << 16)) : i;
-          }
+          if (STATE_SMEM) reinterpret_cast<uint16_t*>(lst + (uint32_t)(r >> 1) * pitch)[r & 1] = (uint16_t)i;
           if (i >= (uint32_t)V) {
             bad = true;
           } else {
@@ -152,13 +153,8 @@ __global__ void __launch_bounds__(256) pe_decode_kernel(PeFwdView f, const uint8
       L1[b2 * pitch] = w1;
       if (w1 == 0u) L2 &= ~(1ull << b2);
     }
-    uint32_t i;
-    if (STATE_SMEM) {
-      const uint32_t pair = lst[(r >> 1) * pitch];
-      i = (r & 1u) ? (pair >> 16) : (pair & 0xFFFFu);
-    } else {
-      i = (uint32_t)list_col[(size_t)r * Ks];
-    }
+    const uint32_t i = STATE_SMEM ? (uint32_t) reinterpret_cast<const uint16_t*>(lst + (r >> 1) * pitch)[r & 1u]
+                                  : (uint32_t)list_col[(size_t)r * Ks];
     order_col[(size_t)k * Ks] = (uint16_t)i;
     const uint32_t e_end = fp.ptr[i + 1];
     for (uint32_t e = fp.ptr[i]; e < e_end; ++e) {   // one predecessor fewer is missing at every successor
