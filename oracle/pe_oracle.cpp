@@ -25,8 +25,18 @@
 // reported as a flag, never repaired (Section III: "valid arrangement").
 //
 // One forward pass in pi order yields that least solution exactly, because pi is a
-// topological order of B joined with the per-machine chains.  Channel exclusivity
-// (Eqs. 14-15) is not applied: communication is a pure delay here.
+// topological order of B joined with the per-machine chains.  By default channel exclusivity
+// (Eqs. 14-15) is not applied: communication is a pure delay.
+//
+// With the flag kCommExclusive the channel (j1 -> j2) carries one transfer at a time
+// (Section III: "each communication channel can only handle one communication task at a
+// time"; Eqs. 14-15).  The paper leaves the sequence of the transfers on a channel to the
+// solver (the variables w); here pi fixes it the way it fixes y: the transfers of a channel
+// follow each other in the order in which their receiving operations appear in pi, and the
+// transfers into one operation in the order of the edge list.  The transfer of edge (i1, i2)
+// then starts at c = max(e_i1 (Eq. 13), end of the previous transfer on its channel (Eq. 14)),
+// ends at d = c + D^c (Eq. 11), and s_i2 >= d (Eq. 12).  Edges inside one machine and edges
+// over a machine pair without a channel move nothing and occupy nothing.
 //
 // Pins (tests/test_oracle_pins.py): exhaustive enumeration on tiny DAGs against a
 // constraint checker, closed forms for uniform pipelines, single-machine prefix sums,
@@ -48,6 +58,7 @@ namespace {
 
 constexpr uint32_t kAssignByPos = 1u;  // `assign` holds x[pi[k]] at row k instead of x[i] at row i
 constexpr uint32_t kTimesByOp = 2u;    // start/finish rows are operations instead of positions
+constexpr uint32_t kCommExclusive = 4u;  // channels carry one transfer at a time (Eqs. 14-15), see below
 
 constexpr uint32_t kStatusAssignRange = 1u;
 constexpr uint32_t kStatusOrderInvalid = 2u;
@@ -80,6 +91,7 @@ extern "C" int pe_oracle_eval(int32_t V, int32_t E, const int32_t* edge_src, con
   std::vector<int32_t> x(V), s(V), e(V), free_at(D), busy_j(D), lvl(D), peak(D);
   std::vector<uint32_t> pi_c(V);
   std::vector<char> done(V);
+  std::vector<int32_t> chan_free((flags & kCommExclusive) ? (size_t)D * D : 0);  // end of the last transfer per channel
 
   for (int64_t c = c_begin; c < c_end; ++c) {
     uint32_t st = 0;
@@ -116,6 +128,7 @@ extern "C" int pe_oracle_eval(int32_t V, int32_t E, const int32_t* edge_src, con
       for (int32_t i = 0; i < V; ++i) lvl[x[i]] += mem_weight[i];
     for (int32_t j = 0; j < D; ++j) peak[j] = lvl[j];
     for (int32_t i = 0; i < V; ++i) { done[i] = 0; s[i] = 0; e[i] = 0; }
+    for (int32_t& v : chan_free) v = 0;
     int32_t z = 0;
 
     for (int32_t k = 0; k < V; ++k) {
@@ -132,8 +145,16 @@ extern "C" int pe_oracle_eval(int32_t V, int32_t E, const int32_t* edge_src, con
         int32_t t = e[p];
         if (x[p] != j) {
           const uint32_t cls = link_class ? link_class[(size_t)x[p] * D + j] : 0u;
-          if (cls == 0xFFu) st |= kStatusNoChannel;  // Eq. 10: no channel between the two machines
-          else t += comm[(size_t)b * L + cls];
+          if (cls == 0xFFu) {
+            st |= kStatusNoChannel;  // Eq. 10: no channel between the two machines
+          } else if (flags & kCommExclusive) {
+            int32_t& chan = chan_free[(size_t)x[p] * D + j];
+            const int32_t c_start = t > chan ? t : chan;           // Eq. 13 and Eq. 14
+            t = c_start + (comm ? comm[(size_t)b * L + cls] : 0);  // Eq. 11
+            chan = t;
+          } else {
+            t += comm ? comm[(size_t)b * L + cls] : 0;
+          }
         }
         if (t > r) r = t;
       }

@@ -19,6 +19,7 @@ _lib = None
 
 ASSIGN_BY_POS = 1
 TIMES_BY_OP = 2
+COMM_EXCLUSIVE = 4
 
 STATUS_ASSIGN_RANGE = 1
 STATUS_ORDER_INVALID = 2

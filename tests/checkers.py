@@ -193,3 +193,56 @@ def critical_path(w):
     dist = bellman_ford(g, directed=True, indices=V)
     starts = -dist[:V] - 1
     return int(np.max(starts + np.asarray(w.dur)))
+
+
+def exclusive_channel_starts(w, x, pi):
+    """Start times under exclusive channels (Eqs. 11-15) as longest-path distances in the explicit
+    constraint graph, by scipy's Bellman-Ford on negated weights.  Nodes: one per operation (its start)
+    and one per cross-machine edge with a channel (the start c of its transfer).  Arcs:
+      machine chain (Eqs. 7-8)   s_next >= s_prev + dur_prev      for consecutive same-machine ops of pi
+      Eq. 13                     c_b    >= s_p + dur_p
+      Eqs. 11-12                 s_i    >= c_b + D^c_b
+      Eq. 14                     c_b'   >= c_b + D^c_b             for consecutive transfers of a channel,
+                                 sequenced by the position of the receiving op in pi, then by edge number
+      same machine / no channel  s_i    >= s_p + dur_p
+    Needs durations and communication times >= 1 (the sparse matrix drops zero weights)."""
+    from scipy.sparse import csr_matrix
+    from scipy.sparse.csgraph import bellman_ford
+    V, E = w.num_ops, w.num_edges
+    pos = np.empty(V, dtype=np.int64)
+    pos[np.asarray(pi)] = np.arange(V)
+    weights = {}
+
+    def add(a, b, wt):
+        assert wt > 0
+        weights[(a, b)] = max(weights.get((a, b), 0), wt)
+
+    last = {}
+    for i in pi:
+        j = int(x[i])
+        if j in last:
+            add(last[j], int(i), int(w.dur[last[j]]))
+        last[j] = int(i)
+    per_channel = {}
+    for b in range(E):
+        p, i = int(w.edge_src[b]), int(w.edge_dst[b])
+        jp, ji = int(x[p]), int(x[i])
+        cls = 0 if w.link_class is None else int(w.link_class[jp, ji])
+        if jp == ji or cls == 0xFF:
+            add(p, i, int(w.dur[p]))
+            continue
+        t = V + 1 + b                                      # node of this edge's transfer
+        add(p, t, int(w.dur[p]))
+        add(t, i, int(w.comm[b, cls]))
+        per_channel.setdefault((jp, ji), []).append((int(pos[i]), b, int(w.comm[b, cls])))
+    for seq in per_channel.values():
+        seq.sort()
+        for (_, b0, c0), (_, b1, _) in zip(seq, seq[1:]):
+            add(V + 1 + b0, V + 1 + b1, c0)
+    n = V + 1 + E
+    rows = [a for a, _ in weights] + [V] * V
+    cols = [b for _, b in weights] + list(range(V))
+    vals = [-float(v) for v in weights.values()] + [-1.0] * V
+    g = csr_matrix((vals, (rows, cols)), shape=(n, n))
+    dist = bellman_ford(g, directed=True, indices=V)
+    return (-dist[:V] - 1).astype(np.int64)
