@@ -81,6 +81,13 @@ int pe_destroy(pe_graph* g);
 enum {
   PE_ASSIGN_BY_POS = 1u, /* `assign` row k holds x[pi[k]] (the machine sequence) instead of row i holding x[i] */
   PE_TIMES_BY_OP = 2u,   /* `start` / `finish` row i belongs to operator i instead of row k to position k */
+  PE_COMM_EXCLUSIVE = 4u, /* a channel (machine j1 -> machine j2) carries one transfer at a time (Section III;
+                            Eqs. 14-15) instead of transfers being pure delays.  The transfers of a channel follow
+                            each other in the order in which their receiving operators appear in pi (as pi fixes y),
+                            those into one operator in the order of the edge list; the transfer of (i1, i2) starts
+                            at max(e_i1, end of the channel's previous transfer) (Eqs. 13, 14), lasts D^c (Eq. 11),
+                            and i2 starts no earlier than its end (Eq. 12).  Runs the global-state kernel only
+                            (PE_VARIANT_AUTO or PE_VARIANT_GLOBAL); needs D*D*K*4 more bytes of workspace. */
   /* Kernel variant (bits 8..11); 0 lets the library choose from (V, E, D, L) and the device. */
   PE_VARIANT_AUTO = 0u << 8,
   PE_VARIANT_GLOBAL = 1u << 8, /* one thread per candidate, finish-time state in the caller's workspace */

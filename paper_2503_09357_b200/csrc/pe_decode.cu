@@ -180,7 +180,9 @@ static bool decode_plan(const pe_graph* g, int64_t K, uint32_t flags, DecodePlan
   if (want == PE_VARIANT_AUTO || want == PE_VARIANT_SHARED) {
     const size_t per = 4 * (V + n0 + n1 + (V + 1) / 2);
     const size_t fixed = (size_t)g->fview.bytes + 16;
-    if (fixed + 32 * per <= g->smem_optin) {
+    // with a single warp per SM the shared-state variant loses to the global-state one (measured at
+    // V = 1024: 3.2e9 against ~7e9 operators/s), so it needs room for two warps unless it was asked for
+    if (fixed + (want == PE_VARIANT_SHARED ? 32 : 64) * per <= g->smem_optin) {
       size_t T = (g->smem_optin - fixed) / per;
       if (T > 256) T = 256;
       T = T / 32 * 32;

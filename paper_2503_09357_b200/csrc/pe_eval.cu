@@ -32,7 +32,7 @@ template <typename OrderT, bool BY_POS>
 __global__ void pe_eval_global_kernel(PeGraphView g, const uint8_t* __restrict__ blob, int64_t K,
                                       const uint8_t* __restrict__ assign, const OrderT* __restrict__ order,
                                       pe_outputs out, uint32_t flags, int32_t* __restrict__ e_state,
-                                      uint8_t* __restrict__ x_state) {
+                                      uint8_t* __restrict__ x_state, int32_t* __restrict__ chan_free) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   int32_t* dev = reinterpret_cast<int32_t*>(smem_raw);
   const int T = blockDim.x;
@@ -71,8 +71,17 @@ __global__ void pe_eval_global_kernel(PeGraphView g, const uint8_t* __restrict__
       if (xp >= (uint32_t)D) xp = D - 1;
       if ((int)xp != j) {
         const uint32_t cl = gp.cls[xp * D + j];
-        if (cl == 0xFFu) st |= PE_STATUS_NO_CHANNEL;
-        else ep += gp.comm[(size_t)q * L + cl];
+        if (cl == 0xFFu) {
+          st |= PE_STATUS_NO_CHANNEL;
+        } else if (chan_free) {
+          // PE_COMM_EXCLUSIVE: the channel (machine of p -> j) carries one transfer at a time; this one starts
+          // when p has ended (Eq. 13) and the channel's previous transfer is through (Eq. 14), lasts D^c (Eq. 11)
+          int32_t* ch = chan_free + (size_t)(xp * D + j) * Ks + c;
+          ep = max(ep, *ch) + gp.comm[(size_t)q * L + cl];
+          *ch = ep;
+        } else {
+          ep += gp.comm[(size_t)q * L + cl];
+        }
       }
       r = max(r, ep);
     }
@@ -293,7 +302,8 @@ static bool plan_warp(const pe_graph* g, int64_t K, uint32_t flags, bool allow_c
 
 static bool plan_global(const pe_graph* g, int64_t K, uint32_t flags, bool allow_compact, Plan* p) {
   p->compact = false;
-  if (g->narrow_ok && allow_compact && g->time_bound < kPackedTimeLimit) {
+  const bool exclusive = (flags & PE_COMM_EXCLUSIVE) != 0;   // only the generic kernel sequences transfers per channel
+  if (!exclusive && g->narrow_ok && allow_compact && g->time_bound < kPackedTimeLimit) {
     // compact-graph kernel with the state in the workspace.  Per-machine records stay in shared
     // memory while a 128-thread block needs at most 16 KB for them; beyond that they would cap the
     // resident candidates, so they move to the workspace too (tiles that stay in L2).
@@ -325,6 +335,8 @@ static bool plan_global(const pe_graph* g, int64_t K, uint32_t flags, bool allow
   p->graph_smem = false;
   p->ws_x_off = round_up((size_t)g->V * (size_t)K * 4, 256);
   p->workspace = p->ws_x_off + ((flags & PE_ASSIGN_BY_POS) ? round_up((size_t)g->V * (size_t)K, 256) : 0);
+  p->ws_c_off = p->workspace;   // PE_COMM_EXCLUSIVE: end of the last transfer per channel, [D*D][K]
+  if (exclusive) p->workspace += round_up((size_t)g->D * g->D * (size_t)K * 4, 256);
   return true;
 }
 
@@ -332,9 +344,13 @@ static bool plan_global(const pe_graph* g, int64_t K, uint32_t flags, bool allow
 // wanted or both absent).  Size queries pass true and false and take the larger workspace.
 static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, bool allow_compact, Plan* p) {
   if (!g || K < 0) return PE_ERR_INVALID_ARG;
-  if (flags & ~(uint32_t)(PE_ASSIGN_BY_POS | PE_TIMES_BY_OP | PE_VARIANT_MASK)) return PE_ERR_INVALID_ARG;
+  if (flags & ~(uint32_t)(PE_ASSIGN_BY_POS | PE_TIMES_BY_OP | PE_COMM_EXCLUSIVE | PE_VARIANT_MASK)) return PE_ERR_INVALID_ARG;
   *p = Plan();
   const uint32_t want = flags & PE_VARIANT_MASK;
+  if (flags & PE_COMM_EXCLUSIVE) {   // exclusive channels: the generic global-state kernel only
+    if (want != PE_VARIANT_AUTO && want != PE_VARIANT_GLOBAL) return PE_ERR_UNSUPPORTED;
+    return plan_global(g, K, flags, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+  }
   switch (want) {
     case PE_VARIANT_AUTO: {
       // Thread-per-candidate with everything on chip wins whenever about a warp and a half of
@@ -384,9 +400,14 @@ static int launch_typed(const pe_graph* g, const Plan& p, int64_t K, const uint8
     int32_t* e_state = static_cast<int32_t*>(workspace);
     uint8_t* x_state = static_cast<uint8_t*>(workspace) + p.ws_x_off;
     if (cudaMemsetAsync(e_state, 0xFF, (size_t)g->V * (size_t)K * 4, stream) != cudaSuccess) return PE_ERR_CUDA;
+    int32_t* chan_free = nullptr;
+    if (flags & PE_COMM_EXCLUSIVE) {
+      chan_free = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + p.ws_c_off);
+      if (cudaMemsetAsync(chan_free, 0, (size_t)g->D * g->D * (size_t)K * 4, stream) != cudaSuccess) return PE_ERR_CUDA;
+    }
     auto kern = pe_eval_global_kernel<OrderT, BY_POS>;
     if (!set_smem(kern, p.smem)) return PE_ERR_CUDA;
-    kern<<<grid, p.threads, p.smem, stream>>>(view, g->d_blob, K, assign, ord, out, flags, e_state, x_state);
+    kern<<<grid, p.threads, p.smem, stream>>>(view, g->d_blob, K, assign, ord, out, flags, e_state, x_state, chan_free);
   } else if (p.variant == PE_VARIANT_SHARED) {
     if (p.graph_smem) {
       auto kern = pe_eval_shared_kernel<OrderT, BY_POS, true>;

@@ -16,6 +16,7 @@ struct Plan {
   bool graph_smem = false;  // graph blob staged into shared memory
   size_t workspace = 0;   // bytes of caller workspace
   size_t ws_x_off = 0;    // offset of the machine-state array inside the workspace (generic GLOBAL, by-pos)
+  size_t ws_c_off = 0;    // generic GLOBAL with PE_COMM_EXCLUSIVE: offset of the per-channel array inside the workspace
   int warp_words = 0;     // WARP: 32-bit words of shared memory per candidate
   bool compact = false;   // SHARED / GLOBAL / WARP: the compact-graph kernels
   bool slab = false;      // WARP (compact): order entries and times go through shared tiles, a slab at a time

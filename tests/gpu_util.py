@@ -44,7 +44,7 @@ def compare(gpu, ref, label=""):
 
 
 def check(graph, w, assign, order, flags=0, want_times=True, label="", threads=None):
-    ref = orc.evaluate(w, assign, order, flags=flags & 3, want_times=want_times, threads=threads or CPU_THREADS)
+    ref = orc.evaluate(w, assign, order, flags=flags & 7, want_times=want_times, threads=threads or CPU_THREADS)
     gpu = gpu_eval(graph, assign, order, flags=flags, want_times=want_times)
     compare(gpu, ref, label)
     return gpu, ref

@@ -1,0 +1,65 @@
+"""Parity of the exclusive-channel communication model (PE_COMM_EXCLUSIVE, Eqs. 14-15) with the oracle."""
+import numpy as np
+import pytest
+
+from paper_2503_09357_b200 import workloads as wl
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pe():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    from paper_2503_09357_b200 import binding
+    return binding
+
+
+CASES = [(1, {}, 1024), (2, {}, 4099), (3, {}, 1031), (4, {}, 2049), (5, dict(V=256, D=64), 2000), (5, dict(V=1024, D=8), 1500)]
+
+
+@pytest.mark.parametrize("config,kw,K", CASES, ids=lambda v: str(v).replace(" ", ""))
+def test_exclusive_channels_match_the_oracle(pe, config, kw, K):
+    w = wl.make_config(config, **kw)
+    assign, order = wl.make_candidates(w, K=K)
+    g = pe.Graph(w)
+    try:
+        assert g.variant(K, pe.PE_COMM_EXCLUSIVE) == "global"
+        gpu, ref = gu.check(g, w, assign, order, flags=pe.PE_COMM_EXCLUSIVE, label=f"exclusive {config} {kw}")
+        plain = gu.gpu_eval(g, assign, order)
+        assert (gpu["finish"] >= plain["finish"]).all()
+        if config >= 3:
+            assert (gpu["makespan"] > plain["makespan"]).any()      # the channels do bind on these workloads
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("layout", ["assign_by_pos", "times_by_op", "summary_only"])
+def test_exclusive_channels_with_layout_flags(pe, layout):
+    w = wl.make_config(3)
+    K = 333
+    assign, order = wl.make_candidates(w, K=K)
+    base = {"assign_by_pos": pe.PE_ASSIGN_BY_POS, "times_by_op": pe.PE_TIMES_BY_OP, "summary_only": 0}[layout]
+    a = wl.assign_by_pos(assign, order) if base & pe.PE_ASSIGN_BY_POS else assign
+    g = pe.Graph(w)
+    try:
+        gu.check(g, w, a, order, flags=base | pe.PE_COMM_EXCLUSIVE, want_times=layout != "summary_only", label=layout)
+    finally:
+        g.close()
+
+
+def test_only_the_global_state_kernel_offers_it(pe):
+    w = wl.make_config(1)
+    g = pe.Graph(w)
+    try:
+        K = 64
+        assert pe.pe_eval_variant(g.handle, K, pe.PE_COMM_EXCLUSIVE | pe.PE_VARIANT_SHARED) == pe.PE_ERR_UNSUPPORTED
+        assert pe.pe_eval_variant(g.handle, K, pe.PE_COMM_EXCLUSIVE | pe.PE_VARIANT_WARP) == pe.PE_ERR_UNSUPPORTED
+        assert pe.pe_eval_variant(g.handle, K, pe.PE_COMM_EXCLUSIVE | pe.PE_VARIANT_GLOBAL) == pe.PE_VARIANT_GLOBAL
+        plain = pe.pe_workspace_bytes(g.handle, K, pe.PE_VARIANT_GLOBAL)
+        assert pe.pe_workspace_bytes(g.handle, K, pe.PE_COMM_EXCLUSIVE) >= w.num_devices ** 2 * K * 4
+        assert plain > 0
+    finally:
+        g.close()
