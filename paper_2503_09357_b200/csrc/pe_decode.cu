@@ -133,35 +133,46 @@ __global__ void __launch_bounds__(256) pe_decode_kernel(PeFwdView f, const uint8
   if (status) status[c] = bad ? (uint32_t)PE_STATUS_ORDER_INVALID : 0u;
   if (bad) return;   // not a permutation: the order of this candidate stays unwritten
 
+  // Main loop.  Every iteration hands one successor of the operator placed last its "one predecessor fewer"
+  // and, once that operator's successor list is used up, places the next operator.  All candidates share the
+  // graph, so every lane needs the same number of successor steps and placements in total; spreading them
+  // over uniform iterations keeps the lanes of a warp busy where a loop over each operator's successors
+  // would make the whole warp wait for the lane that drew the operator with the most successors.
   uint16_t* order_col = order + c;
-  for (int k = 0; k < V; ++k) {
-    if (L2 == 0) break;   // cannot happen for a permutation over a DAG; keeps the loop in bounds regardless
-    // the smallest available rank: first set bit of each level, top down
-    const uint32_t b2 = (uint32_t)__ffsll((long long)L2) - 1u;
-    uint32_t w1 = L1[b2 * pitch];
-    if (w1 == 0u) break;   // (a summary bit without anything below it: cannot happen either)
-    const uint32_t b1 = (uint32_t)__ffs((int)w1) - 1u;
-    const uint32_t i0 = b2 * 32u + b1;
-    uint32_t w0 = L0[i0 * pitch];
-    if (w0 == 0u) break;
-    const uint32_t b0 = (uint32_t)__ffs((int)w0) - 1u;
-    const uint32_t r = i0 * 32u + b0;
-    w0 &= ~(1u << b0);
-    L0[i0 * pitch] = w0;
-    if (w0 == 0u) {
-      w1 &= ~(1u << b1);
-      L1[b2 * pitch] = w1;
-      if (w1 == 0u) L2 &= ~(1ull << b2);
-    }
-    const uint32_t i = STATE_SMEM ? (uint32_t) reinterpret_cast<const uint16_t*>(lst + (r >> 1) * pitch)[r & 1u]
-                                  : (uint32_t)list_col[(size_t)r * Ks];
-    order_col[(size_t)k * Ks] = (uint16_t)i;
-    const uint32_t e_end = fp.ptr[i + 1];
-    for (uint32_t e = fp.ptr[i]; e < e_end; ++e) {   // one predecessor fewer is missing at every successor
-      const uint32_t s = fp.succ[e];
+  uint32_t e = 0, e_end = 0;
+  int k = 0;
+  for (int it = 0; it < 2 * V + f.E + 2; ++it) {   // (bound: at most V placements and E successor steps)
+    if (e < e_end) {
+      const uint32_t s = fp.succ[e++];
       const uint32_t w = word[s * pitch] - (1u << 16);
       word[s * pitch] = w;
       if (((w >> 16) & 0xFFu) == 0u) add(w & 0xFFFFu);
+    }
+    if (e == e_end) {
+      if (k == V || L2 == 0) break;   // all placed (L2 == 0 earlier cannot happen for a permutation over a DAG)
+      // the smallest available rank: first set bit of each level, top down
+      const uint32_t b2 = (uint32_t)__ffsll((long long)L2) - 1u;
+      uint32_t w1 = L1[b2 * pitch];
+      if (w1 == 0u) break;   // (a summary bit without anything below it: cannot happen either)
+      const uint32_t b1 = (uint32_t)__ffs((int)w1) - 1u;
+      const uint32_t i0 = b2 * 32u + b1;
+      uint32_t w0 = L0[i0 * pitch];
+      if (w0 == 0u) break;
+      const uint32_t b0 = (uint32_t)__ffs((int)w0) - 1u;
+      const uint32_t r = i0 * 32u + b0;
+      w0 &= ~(1u << b0);
+      L0[i0 * pitch] = w0;
+      if (w0 == 0u) {
+        w1 &= ~(1u << b1);
+        L1[b2 * pitch] = w1;
+        if (w1 == 0u) L2 &= ~(1ull << b2);
+      }
+      const uint32_t i = STATE_SMEM ? (uint32_t) reinterpret_cast<const uint16_t*>(lst + (r >> 1) * pitch)[r & 1u]
+                                    : (uint32_t)list_col[(size_t)r * Ks];
+      order_col[(size_t)k * Ks] = (uint16_t)i;
+      ++k;
+      e = fp.ptr[i];
+      e_end = fp.ptr[i + 1];
     }
   }
 }
