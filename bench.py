@@ -46,6 +46,7 @@ KERNEL_OF_VARIANT = {"shared": "pe_eval_lane_kernel<STATE_SMEM=true>", "global":
 NCU_TRAFFIC = {
     # variant: (hash of csrc/ at capture time, DRAM bytes per operator-evaluation, captured workload)
     "global": ("0422252154d12689", 370.0, "random_layered_V16384_D64 at K = 32768 (half size), scaled by operator-evaluations"),
+    "warp": ("726a662187ccfe26", 10.53, "random_layered_V16384_D64 at K = 4096, scaled by operator-evaluations"),
 }
 
 
@@ -170,6 +171,34 @@ def run_reference(args):
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+def time_decode(pe, name, dev, local_rank, stream, op_budget, steps=5):
+    """pe_decode_priority on uniformly random priority lists of one workload (made on the device: argsort of
+    random numbers per candidate), K * V about `op_budget`; mean of `steps` timed calls after two warm-ups."""
+    import torch
+    ow = WORKLOADS[name]()
+    oV = ow.num_ops
+    oK = int(min(ow.num_candidates, max(1024, op_budget // oV)))
+    og = pe.Graph(ow, device=local_rank)
+    gen = torch.Generator(device=dev); gen.manual_seed(oV)
+    plist = torch.argsort(torch.rand((oV, oK), device=dev, generator=gen), dim=0).to(torch.int16).contiguous()
+    for _ in range(2):
+        og.decode_priority(plist)
+    torch.cuda.synchronize(dev)
+    times = []
+    for _ in range(steps):
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream); dorder, dstatus = og.decode_priority(plist); e1.record(stream)
+        torch.cuda.synchronize(dev)
+        times.append(e0.elapsed_time(e1))
+    ms = statistics.mean(times)
+    assert int(dstatus.abs().max()) == 0
+    dalg = oK * oV * 4 + oK * 4                    # list in, order out, status
+    rec = {"workload": name, "V": oV, "K": oK, "kernel_variant": pe.VARIANT_NAMES[pe.pe_decode_variant(og.handle, oK, 0)],
+           "ms": ms, "op_decodes_per_s": oK * oV / (ms * 1e-3), "gbs": dalg / (ms * 1e-3) / 1e9}
+    og.close()
+    return rec
 
 
 def run_ours(args):
@@ -320,36 +349,11 @@ def run_ours(args):
             og.close()
             del da, do, oout, ows
             torch.cuda.empty_cache()
-        # the step in front of the path: priority-list decoding, on uniformly random lists (device-made:
-        # argsort of random numbers per candidate), K * V = 2^28 per workload
-        decode = []
+        # the step in front of the path: priority-list decoding, K * V = 2^28 per workload
         for name in sorted(WORKLOADS):
             if name.endswith("_D64") or name == "tiny_pipeline":
                 continue                                  # decoding does not depend on the machines
-            ow = WORKLOADS[name]()
-            oV = ow.num_ops
-            oK = int(min(ow.num_candidates, max(1024, (1 << 28) // oV)))
-            og = pe.Graph(ow, device=local_rank)
-            gen = torch.Generator(device=dev); gen.manual_seed(oV)
-            plist = torch.argsort(torch.rand((oV, oK), device=dev, generator=gen), dim=0).to(torch.int16).contiguous()
-            for _ in range(2):
-                og.decode_priority(plist)
-            torch.cuda.synchronize(dev)
-            times = []
-            for _ in range(5):
-                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-                e0.record(stream); dorder, dstatus = og.decode_priority(plist); e1.record(stream)
-                torch.cuda.synchronize(dev)
-                times.append(e0.elapsed_time(e1))
-            ms = statistics.mean(times)
-            assert int(dstatus.abs().max()) == 0
-            dalg = oK * oV * 4 + oK * 4                    # list in, order out, status
-            decode.append({"workload": name, "V": oV, "K": oK,
-                           "kernel_variant": pe.VARIANT_NAMES[pe.pe_decode_variant(og.handle, oK, 0)], "ms": ms,
-                           "op_decodes_per_s": oK * oV / (ms * 1e-3), "gbs": dalg / (ms * 1e-3) / 1e9})
-            og.close()
-            del plist, dorder, dstatus
-            torch.cuda.empty_cache()
+            decode.append(time_decode(pe, name, dev, local_rank, stream, 1 << 28))
 
     if rank == 0:
         peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -417,10 +421,19 @@ def main():
                     help="skip the device-resident timing of every other configuration (other_workloads); "
                          "it runs by default on 1 GPU and adds about a minute")
     ap.add_argument("--all-workloads", dest="all_workloads", action="store_true", help=argparse.SUPPRESS)
+    ap.add_argument("--decode-only", action="store_true",
+                    help="time pe_decode_priority alone on --workload (K * V = 2^26) and print its record")
     ap.set_defaults(all_workloads=True)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.decode_only:
+        import torch
+        from paper_2503_09357_b200 import binding as pe
+        torch.cuda.set_device(0)
+        print(json.dumps(time_decode(pe, args.workload, torch.device("cuda", 0), 0, torch.cuda.current_stream(), 1 << 26)),
+              flush=True)
+        return
     if args.impl == "reference":
         args.steps = args.steps if args.steps > 0 else 5
         run_reference(args)
