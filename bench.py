@@ -201,6 +201,35 @@ def time_decode(pe, name, dev, local_rank, stream, op_budget, steps=5):
     return rec
 
 
+def time_exclusive(pe, name, dev, local_rank, stream, op_budget, want_times, steps=5):
+    """pe_eval_batch with PE_COMM_EXCLUSIVE (one transfer per channel at a time) on the first K candidates of a
+    workload, K * V about `op_budget`; same compulsory bytes as the plain evaluation."""
+    import torch
+    ow = WORKLOADS[name]()
+    oV, oD = ow.num_ops, ow.num_devices
+    oK = int(min(ow.num_candidates, max(1024, op_budget // oV)))
+    oa, oo = wl.make_candidates(ow, K=oK)
+    og = pe.Graph(ow, device=local_rank)
+    flags = pe.PE_COMM_EXCLUSIVE
+    da = torch.from_numpy(oa).to(dev); do = torch.from_numpy(oo.view(np.int16)).to(dev)
+    oout = og.alloc_outputs(oK, want_times)
+    ows = og.alloc_workspace(oK, flags)
+    for _ in range(2):
+        og.eval_batch(da, do, flags=flags, out=oout, workspace=ows)
+    torch.cuda.synchronize(dev)
+    times = []
+    for _ in range(steps):
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream); og.eval_batch(da, do, flags=flags, out=oout, workspace=ows); e1.record(stream)
+        torch.cuda.synchronize(dev)
+        times.append(e0.elapsed_time(e1))
+    ms = statistics.mean(times)
+    rec = {"workload": name, "V": oV, "D": oD, "K": oK, "kernel_variant": og.variant(oK, flags), "ms": ms,
+           "op_evals_per_s": oK * oV / (ms * 1e-3), "gbs": compulsory_bytes(oV, oD, oK, 2, want_times) / (ms * 1e-3) / 1e9}
+    og.close()
+    return rec
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -316,6 +345,7 @@ def run_ours(args):
 
     others = None
     decode = []
+    exclusive = []
     if rank == 0 and world == 1 and args.all_workloads:
         # free the headline's buffers, then time every other configuration (device-resident, fewer steps)
         del d_assign, d_order, d_out, ws, h_out, houts, outs
@@ -354,6 +384,9 @@ def run_ours(args):
             if name.endswith("_D64") or name == "tiny_pipeline":
                 continue                                  # decoding does not depend on the machines
             decode.append(time_decode(pe, name, dev, local_rank, stream, 1 << 28))
+        # the model variant with exclusive channels (Eqs. 14-15), K * V = 2^26 per workload
+        for name in ("bidirectional_pipeline", "multimodal_mimo", "random_layered_V256_D8", "random_layered_V4096_D64"):
+            exclusive.append(time_exclusive(pe, name, dev, local_rank, stream, 1 << 26, want_times))
 
     if rank == 0:
         peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -397,6 +430,9 @@ def run_ours(args):
             for o in decode:
                 o["frac"] = o["gbs"] / peak
             line["decode"] = decode
+            for o in exclusive:
+                o["frac"] = o["gbs"] / peak
+            line["exclusive_channels"] = exclusive
         print(json.dumps(line), flush=True)
     g.close()
     if world > 1:

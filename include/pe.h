@@ -86,8 +86,9 @@ enum {
                             each other in the order in which their receiving operators appear in pi (as pi fixes y),
                             those into one operator in the order of the edge list; the transfer of (i1, i2) starts
                             at max(e_i1, end of the channel's previous transfer) (Eqs. 13, 14), lasts D^c (Eq. 11),
-                            and i2 starts no earlier than its end (Eq. 12).  Runs the global-state kernel only
-                            (PE_VARIANT_AUTO or PE_VARIANT_GLOBAL); needs D*D*K*4 more bytes of workspace. */
+                            and i2 starts no earlier than its end (Eq. 12).  Offered by the shared-state kernel (no
+                            workspace) and the global-state kernel (D*D*K*4 more bytes of workspace), not by
+                            PE_VARIANT_WARP; ask pe_workspace_bytes with the same flags. */
   /* Kernel variant (bits 8..11); 0 lets the library choose from (V, E, D, L) and the device. */
   PE_VARIANT_AUTO = 0u << 8,
   PE_VARIANT_GLOBAL = 1u << 8, /* one thread per candidate, finish-time state in the caller's workspace */

@@ -214,11 +214,15 @@ __global__ void pe_eval_shared_kernel(PeGraphView g, const uint8_t* __restrict__
 
 static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-static bool plan_shared(const pe_graph* g, bool allow_compact, Plan* p) {
+// exclusive: PE_COMM_EXCLUSIVE - the compact kernel keeps one more word per machine pair and candidate;
+// the generic shared-state kernel does not offer it.
+static bool plan_shared(const pe_graph* g, bool allow_compact, Plan* p, bool exclusive = false) {
   if (g->time_bound >= kPackedTimeLimit) return false;
   p->compact = false;
+  p->exclusive = exclusive;
   if (g->narrow_ok && allow_compact) {  // compact graph staged in shared memory next to the state
-    const size_t per = (size_t)4 * (g->V + 1) + (size_t)(g->has_weight ? 20 : 16) * g->D;
+    const size_t per = (size_t)4 * (g->V + 1) + (size_t)(g->has_weight ? 20 : 16) * g->D +
+                       (exclusive ? (size_t)4 * g->D * g->D : 0);
     const size_t fixed = (size_t)g->nview.bytes + 16;
     if (fixed + 32 * per <= g->smem_optin) {
       // A block size that is a multiple of 32 keeps every lane's state column in its own bank.  That is
@@ -237,6 +241,7 @@ static bool plan_shared(const pe_graph* g, bool allow_compact, Plan* p) {
       return true;
     }
   }
+  if (exclusive) return false;
   const size_t per_thread = (size_t)4 * g->V + (size_t)(g->has_weight ? 20 : 16) * g->D;
   const size_t budget = g->smem_optin;
   for (int with_graph = 1; with_graph >= 0; --with_graph) {
@@ -347,7 +352,14 @@ static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, bool allow_co
   if (flags & ~(uint32_t)(PE_ASSIGN_BY_POS | PE_TIMES_BY_OP | PE_COMM_EXCLUSIVE | PE_VARIANT_MASK)) return PE_ERR_INVALID_ARG;
   *p = Plan();
   const uint32_t want = flags & PE_VARIANT_MASK;
-  if (flags & PE_COMM_EXCLUSIVE) {   // exclusive channels: the generic global-state kernel only
+  if (flags & PE_COMM_EXCLUSIVE) {
+    // exclusive channels: the compact shared-state kernel where a block of candidates still fits with one
+    // more word per machine pair each, else the generic global-state kernel
+    if (want == PE_VARIANT_AUTO || want == PE_VARIANT_SHARED) {
+      if (plan_shared(g, allow_compact, p, true) && (p->threads >= 48 || want == PE_VARIANT_SHARED)) return PE_OK;
+      if (want == PE_VARIANT_SHARED) return PE_ERR_UNSUPPORTED;
+      *p = Plan();
+    }
     if (want != PE_VARIANT_AUTO && want != PE_VARIANT_GLOBAL) return PE_ERR_UNSUPPORTED;
     return plan_global(g, K, flags, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
   }

@@ -53,7 +53,9 @@ __device__ __forceinline__ NarrowPtrs narrow_ptrs(const uint8_t* base, const PeN
 // TIMES: start and finish are both written (true) or both absent (false).
 // DEPTH (one link class only): 3 = no operator has more than three incoming edges, so the three inline
 // slots are all there is and the step is straight-line code; 0 = general (inline slots, then the list).
-template <typename IdxT, bool BY_POS, int CLS, bool STATE_SMEM, bool TIMES, int DEPTH>
+// EXCL (shared-state only): channels carry one transfer at a time (PE_COMM_EXCLUSIVE; Eqs. 14-15): the end of the
+// last transfer per channel sits in shared memory as [machine pair][thread] behind the operator state.
+template <typename IdxT, bool BY_POS, int CLS, bool STATE_SMEM, bool TIMES, int DEPTH, bool EXCL = false>
 __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const uint8_t* __restrict__ nblob, int64_t K,
                                                            const uint8_t* __restrict__ assign,
                                                            const uint16_t* __restrict__ order, pe_outputs out,
@@ -92,6 +94,9 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
   uint32_t* state = STATE_SMEM ? reinterpret_cast<uint32_t*>(sm + (size_t)D * T * 16 + wsum_bytes) + t
                                : gstate + (size_t)(c >> 5) * (size_t)(V + 1) * 32 + (c & 31);
   const uint32_t pitch = STATE_SMEM ? (uint32_t)T : 32u;
+  // EXCL: end of the last transfer on channel (j1 -> j2) at chan[(j1 * D + j2) * T]
+  int32_t* chan = reinterpret_cast<int32_t*>(sm + (size_t)D * T * 16 + wsum_bytes + (size_t)(V + 1) * T * 4) + t;
+  static_assert(!EXCL || STATE_SMEM, "exclusive channels are kept in shared memory");
 
   const uint16_t* order_col = order + c;
   const uint8_t* assign_col = assign + c;
@@ -119,6 +124,8 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
     dev[j * dpitch] = make_int4(0, 0, 0, 0);
     if (gp.weight) wsum[j * dpitch] = 0;
   }
+  if (EXCL)
+    for (int q = 0; q < D * D; ++q) chan[(uint32_t)q * (uint32_t)T] = 0;
   const bool by_op_times = (flags & PE_TIMES_BY_OP) != 0;
   const bool deep = g.max_indeg > 2;
   const uint32_t vmax = (uint32_t)(V - 1), dmax = (uint32_t)(D - 1);
@@ -169,14 +176,27 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
       const uint32_t w = state[p * pitch];
       pred_max = max(pred_max, w);
       const int xp = (int)(w & 0xFFu);
+      const uint32_t xpc = min((uint32_t)xp, dmax);  // (an unscheduled source of an invalid order may still carry a raw id)
       uint32_t delay = lo >> 16;
+      bool channel = true;
       if (NEED_CLS) {
-        const uint32_t cl = gp.cls[xp * D + j];
+        const uint32_t cl = gp.cls[xpc * D + j];
         if (TWO_CLASS) delay = cl == 1u ? hi : delay;
         if (cl == 0xFFu) {
           delay = 0;
+          channel = false;
           if (p != (uint32_t)V && xp != j) st |= PE_STATUS_NO_CHANNEL;
         }
+      }
+      if (EXCL) {
+        // the transfer starts when its source has ended (Eq. 13) and the channel is free (Eq. 14), lasts D^c (Eq. 11)
+        if (xp != j && p != (uint32_t)V && channel) {
+          int32_t* ch = chan + (xpc * D + j) * (uint32_t)T;
+          const int32_t t_end = max((int32_t)(w >> 8), *ch) + (int32_t)delay;
+          *ch = t_end;
+          return t_end;
+        }
+        return (int32_t)(w >> 8);
       }
       return (int32_t)(w >> 8) + (xp != j ? (int32_t)delay : 0);
     };
@@ -187,7 +207,9 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
         for (int q = 1; q < indeg; ++q) r = max(r, edge_time(ed[q].x, ed[q].y));
       }
     } else if (DEPTH == 3) {
-      r = max(r, max(edge_time(rec.w, 0u), edge_time(rec.x, 0u)));
+      const int32_t t1 = edge_time(rec.w, 0u);   // in edge-list order: with EXCL the order of the transfers matters
+      const int32_t t2 = edge_time(rec.x, 0u);
+      r = max(r, max(t1, t2));
     } else {
       r = max(r, edge_time(rec.w, 0u));
       if (deep) {  // some operator has more than two incoming edges: third inline slot, then the CSR list

@@ -172,7 +172,7 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
         const uint32_t xp = w & 0xFFu;
         uint32_t delay = lo >> 16;
         if (NEED_CLS) {
-          const uint32_t cl = gp.cls[xp * D + j];
+          const uint32_t cl = gp.cls[min(xp, dmax) * D + j];  // (an unscheduled source of an invalid order may carry a raw id)
           if (TWO_CLASS) delay = cl == 1u ? hi : delay;
           if (cl == 0xFFu) {
             delay = 0;
@@ -274,7 +274,7 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
         const uint32_t xp = w & 0xFFu;
         uint32_t delay = lo >> 16;
         if (NEED_CLS) {
-          const uint32_t cl = gp.cls[xp * D + j];
+          const uint32_t cl = gp.cls[min(xp, dmax) * D + j];  // (an unscheduled source of an invalid order may carry a raw id)
           if (TWO_CLASS) delay = cl == 1u ? hi : delay;
           if (cl == 0xFFu) {
             delay = 0;

@@ -17,6 +17,11 @@ static int launch4(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* a
                                                gdev);
     return PE_OK;
   };
+  if constexpr (STATE_SMEM) {
+    if (p.exclusive)
+      return out.start ? go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, true, true, DEPTH, true>)
+                       : go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, true, false, DEPTH, true>);
+  }
   return out.start ? go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, true, DEPTH>)
                    : go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, false, DEPTH>);
 }

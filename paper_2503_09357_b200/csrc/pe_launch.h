@@ -19,6 +19,7 @@ struct Plan {
   size_t ws_c_off = 0;    // generic GLOBAL with PE_COMM_EXCLUSIVE: offset of the per-channel array inside the workspace
   int warp_words = 0;     // WARP: 32-bit words of shared memory per candidate
   bool compact = false;   // SHARED / GLOBAL / WARP: the compact-graph kernels
+  bool exclusive = false; // SHARED (compact): PE_COMM_EXCLUSIVE, one more word per machine pair and candidate
   bool slab = false;      // WARP (compact): order entries and times go through shared tiles, a slab at a time
 };
 

@@ -26,8 +26,13 @@ def test_exclusive_channels_match_the_oracle(pe, config, kw, K):
     assign, order = wl.make_candidates(w, K=K)
     g = pe.Graph(w)
     try:
-        assert g.variant(K, pe.PE_COMM_EXCLUSIVE) == "global"
-        gpu, ref = gu.check(g, w, assign, order, flags=pe.PE_COMM_EXCLUSIVE, label=f"exclusive {config} {kw}")
+        seen = set()
+        for name, bit in (("auto", 0), ("shared", pe.PE_VARIANT_SHARED), ("global", pe.PE_VARIANT_GLOBAL)):
+            if pe.pe_eval_variant(g.handle, K, pe.PE_COMM_EXCLUSIVE | bit) < 0:
+                continue
+            gpu, ref = gu.check(g, w, assign, order, flags=pe.PE_COMM_EXCLUSIVE | bit, label=f"exclusive {config} {kw} {name}")
+            seen.add(g.variant(K, pe.PE_COMM_EXCLUSIVE | bit))
+        assert "global" in seen and (config not in (1, 2) or "shared" in seen)
         plain = gu.gpu_eval(g, assign, order)
         assert (gpu["finish"] >= plain["finish"]).all()
         if config >= 3:
@@ -48,18 +53,27 @@ def test_exclusive_channels_with_layout_flags(pe, layout):
         gu.check(g, w, a, order, flags=base | pe.PE_COMM_EXCLUSIVE, want_times=layout != "summary_only", label=layout)
     finally:
         g.close()
+    w = wl.make_config(2)                                    # small enough for the shared-state kernel
+    assign, order = wl.make_candidates(w, K=K)
+    a = wl.assign_by_pos(assign, order) if base & pe.PE_ASSIGN_BY_POS else assign
+    g = pe.Graph(w)
+    try:
+        assert g.variant(K, base | pe.PE_COMM_EXCLUSIVE) == "shared"
+        gu.check(g, w, a, order, flags=base | pe.PE_COMM_EXCLUSIVE, want_times=layout != "summary_only", label=layout + " shared")
+    finally:
+        g.close()
 
 
-def test_only_the_global_state_kernel_offers_it(pe):
+def test_which_kernels_offer_it(pe):
     w = wl.make_config(1)
     g = pe.Graph(w)
     try:
         K = 64
-        assert pe.pe_eval_variant(g.handle, K, pe.PE_COMM_EXCLUSIVE | pe.PE_VARIANT_SHARED) == pe.PE_ERR_UNSUPPORTED
+        assert pe.pe_eval_variant(g.handle, K, pe.PE_COMM_EXCLUSIVE | pe.PE_VARIANT_SHARED) == pe.PE_VARIANT_SHARED
         assert pe.pe_eval_variant(g.handle, K, pe.PE_COMM_EXCLUSIVE | pe.PE_VARIANT_WARP) == pe.PE_ERR_UNSUPPORTED
         assert pe.pe_eval_variant(g.handle, K, pe.PE_COMM_EXCLUSIVE | pe.PE_VARIANT_GLOBAL) == pe.PE_VARIANT_GLOBAL
-        plain = pe.pe_workspace_bytes(g.handle, K, pe.PE_VARIANT_GLOBAL)
+        assert pe.pe_workspace_bytes(g.handle, K, pe.PE_COMM_EXCLUSIVE | pe.PE_VARIANT_GLOBAL) >= w.num_devices ** 2 * K * 4
+        # the size query covers every form of the call (e.g. 32-bit orders, which take the global-state kernel)
         assert pe.pe_workspace_bytes(g.handle, K, pe.PE_COMM_EXCLUSIVE) >= w.num_devices ** 2 * K * 4
-        assert plain > 0
     finally:
         g.close()
