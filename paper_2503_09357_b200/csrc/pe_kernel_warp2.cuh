@@ -14,7 +14,9 @@
 //     (lane, delay) pairs in registers and the window is relaxed with shuffles: every lane
 //     repeatedly takes the maximum of what it has and its sources' current end times plus
 //     delays and ends D^o later (Eq. 3); the values rise to the window's longest-path solution
-//     and the loop stops when nothing changes - mostly long before the window's depth;
+//     and the loop stops when nothing changes - mostly long before the window's depth (used with
+//     many warps per SM; with few, a lane instead evaluates once, when the lanes it waits for are
+//     final, which keeps the loop-carried chain to a ballot and a mask test);
 //   otherwise: the remembered sources are operator ids (the inline ones) or the edge list
 //     itself, the lanes waited for form a mask `need`, and the window is resolved in rounds: a
 //     lane whose `need` lanes have finished evaluates once, from the state in shared memory, and
@@ -163,7 +165,6 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
       // previous operator of the machine inside the window (Eqs. 7-8) is a fourth slot with delay 0.
       constexpr int32_t kNever = -(1 << 29);   // delay of an empty slot: never wins the maximum
       int32_t r_base = 0;
-      int nslots = 0;
       uint32_t depmask = 0;   // lanes of this window this operator waits for
       int l0 = lane, l1 = lane, l2 = lane;
       int32_t d0 = kNever, d1 = kNever, d2 = kNever;
@@ -181,7 +182,8 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
         }
         return xp != j ? delay : 0u;
       };
-      auto classify = [&](uint32_t lo, uint32_t hi) {
+      // edge number q of an operator owns slot q (at most three incoming edges here)
+      auto classify = [&](uint32_t lo, uint32_t hi, int& l_slot, int32_t& d_slot) {
         const uint32_t p = lo & 0xFFFFu;
         const uint32_t w = state[p];
         const uint32_t dly = delay_of(lo, hi, w);
@@ -190,10 +192,8 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
         } else {
           const uint32_t l = (w >> 8) & 31u;
           if (w < kInWindowEnd && l < (uint32_t)lane) {
-            if (nslots == 0) { l0 = (int)l; d0 = (int32_t)dly; }
-            else if (nslots == 1) { l1 = (int)l; d1 = (int32_t)dly; }
-            else if (nslots == 2) { l2 = (int)l; d2 = (int32_t)dly; }
-            ++nslots;
+            l_slot = (int)l;
+            d_slot = (int32_t)dly;
             depmask |= 1u << l;
           } else {
             st |= PE_STATUS_ORDER_INVALID;  // a predecessor that is not before this operator
@@ -203,17 +203,14 @@ __global__ void __launch_bounds__(1024) pe_eval_warp2_kernel(PeNarrowView g, con
       int lp = lane;
       int32_t dp = kNever;
       if (act) {
-        classify(rec.z, rec.w);
+        classify(rec.z, rec.w, l0, d0);
         if (TWO_CLASS) {
           const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
-          for (int q = 1; q < indeg; ++q) classify(ed[q].x, ed[q].y);
+          if (indeg > 1) classify(ed[1].x, ed[1].y, l1, d1);
+          if (indeg > 2) classify(ed[2].x, ed[2].y, l2, d2);
         } else {
-          classify(rec.w, 0u);
-          classify(third, 0u);
-          if (!FLAT && indeg > 3) {
-            const uint32_t* ed = gp.edges + rec.x;
-            for (int q = 2; q < indeg; ++q) classify(ed[q], 0u);
-          }
+          classify(rec.w, 0u, l1, d1);
+          classify(rec.x, 0u, l2, d2);
         }
         if (prev < 0) r_base = max(r_base, free_at[j]);
         else { lp = prev; dp = 0; depmask |= 1u << prev; }   // Eqs. 7-8: after the machine's previous operator
