@@ -77,3 +77,24 @@ def test_one_machine_and_missing_channels_move_nothing():
     w.link_class = np.full((w.num_devices, w.num_devices), 0xFF, np.uint8)
     a = orc.evaluate(w, assign, order, flags=orc.COMM_EXCLUSIVE); b = orc.evaluate(w, assign, order)
     assert np.array_equal(a["finish"], b["finish"]) and (a["status"] & orc.STATUS_NO_CHANNEL).any()
+
+
+def test_golden_worked_example_exclusive_channels_and_decoding():
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "worked_example_exclusive_channels_and_decoding.txt")
+    edges, comm = [(0, 2), (1, 2), (0, 3), (2, 4), (3, 4)], [[2], [1], [5], [3], [1]]
+    w = ck.problem(5, edges, [3, 2, 4, 1, 2], 2, comm=comm)
+    ints = lambda s: [int(t) for t in s.split()]
+    rows = [l for l in open(path) if l.strip() and l[0] != "#"]
+    assert [r[0] for r in rows] == ["E", "E", "P", "P", "P"]
+    for line in rows:
+        f = [x.strip() for x in line.split("|")]
+        if f[0] == "E":
+            x, pi, s, e, z = [ints(t) for t in f[1:]]
+            assign, order = ck.columns([x], [pi], 5)
+            out = orc.evaluate(w, assign, order, flags=orc.COMM_EXCLUSIVE | orc.TIMES_BY_OP)
+            assert out["start"][:, 0].tolist() == s and out["finish"][:, 0].tolist() == e and int(out["makespan"][0]) == z[0]
+        else:
+            lst, expect = ints(f[1]), ints(f[2])
+            dec, status = orc.decode(w, np.array(lst, np.uint16)[:, None])
+            assert status[0] == 0 and dec[:, 0].tolist() == expect
