@@ -218,6 +218,13 @@ int pe_select_best(int64_t K, const int32_t* makespan, const uint32_t* status, u
  * PE_ERR_TIMEOUT if a kernel gave up a bounded wait (its outputs are then invalid).  Clears the word. */
 int pe_graph_poll_error(pe_graph* g, void* cuda_stream);
 
+/* Self-test of the library's bounded device-side wait (the only wait its kernels have is the one for the
+ * bulk copy that stages the graph into shared memory): launches one small block whose barrier expects bytes
+ * that no copy brings, so the wait runs out after 1024 polls, the block sets the graph's error word and
+ * returns.  Nothing faults and nothing stays in flight; a following pe_graph_poll_error returns
+ * PE_ERR_TIMEOUT once and the graph remains usable.  Asynchronous on `cuda_stream`. */
+int pe_selftest_wait_timeout(pe_graph* g, void* cuda_stream);
+
 /* Number of kernels this library has launched in this process so far (all graphs, all streams). */
 int64_t pe_kernel_launches(void);
 

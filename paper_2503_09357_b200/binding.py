@@ -73,6 +73,8 @@ _lib.pe_select_best.restype = ctypes.c_int
 _lib.pe_select_best.argtypes = [ctypes.c_int64, _P, _P, ctypes.c_uint32, _P, _P]
 _lib.pe_graph_poll_error.restype = ctypes.c_int
 _lib.pe_graph_poll_error.argtypes = [_P, _P]
+_lib.pe_selftest_wait_timeout.restype = ctypes.c_int
+_lib.pe_selftest_wait_timeout.argtypes = [_P, _P]
 _lib.pe_kernel_launches.restype = ctypes.c_int64
 _lib.pe_kernel_launches.argtypes = []
 _lib.pe_strerror.restype = ctypes.c_char_p
@@ -198,6 +200,10 @@ def pe_decode_priority(handle, K, list_ptr, order_bytes, flags, order_ptr, statu
 
 def pe_graph_poll_error(handle, stream=0) -> int:
     return _lib.pe_graph_poll_error(handle, stream or None)
+
+
+def pe_selftest_wait_timeout(handle, stream=0) -> int:
+    return _lib.pe_selftest_wait_timeout(handle, stream or None)
 
 
 def pe_kernel_launches() -> int:

@@ -76,8 +76,8 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 // Bounded wait: gives up after kWaitLimit polls (each poll may itself block for a short,
 // hardware-defined time) and reports it instead of spinning for ever.
 constexpr int kWaitLimit = 1 << 20;
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-  for (int it = 0; it < kWaitLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, int limit = kWaitLimit) {
+  for (int it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (it > 32) __nanosleep(64);
   }

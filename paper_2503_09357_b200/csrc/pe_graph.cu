@@ -5,6 +5,7 @@
 #include <new>
 #include <vector>
 
+#include "pe_device.cuh"
 #include "pe_graph.h"
 
 namespace {
@@ -288,6 +289,28 @@ extern "C" int pe_graph_poll_error(pe_graph* g, void* cuda_stream) {
   if (cudaMemcpy(&word, g->d_error, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PE_ERR_CUDA;
   if (word != 0 && cudaMemset(g->d_error, 0, sizeof(int)) != cudaSuccess) return PE_ERR_CUDA;
   return word;
+}
+
+// Self-test of the bounded wait: the barrier is told to expect bytes that no copy will ever bring, so the
+// wait runs out after `limit` polls, the error word is set and the block returns - nothing is in flight.
+__global__ void pe_selftest_wait_kernel(int* err, int limit) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) pe::mbar_init(&bar, 1);
+  __syncthreads();
+  if (threadIdx.x == 0) pe::mbar_expect_tx(&bar, 16);
+  __syncthreads();
+  if (!pe::mbar_wait_bounded(&bar, 0, limit)) atomicExch(err, PE_ERR_TIMEOUT);
+}
+
+extern "C" int pe_selftest_wait_timeout(pe_graph* g, void* cuda_stream) {
+  if (!g) return PE_ERR_INVALID_ARG;
+  int prev = -1;
+  if (cudaGetDevice(&prev) != cudaSuccess) return PE_ERR_CUDA;
+  if (prev != g->device && cudaSetDevice(g->device) != cudaSuccess) return PE_ERR_CUDA;
+  pe_selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)cuda_stream>>>(g->d_error, 1024);
+  const int ret = cudaGetLastError() == cudaSuccess ? PE_OK : PE_ERR_CUDA;
+  if (prev != g->device) cudaSetDevice(prev);
+  return ret;
 }
 
 extern "C" const char* pe_strerror(int code) {

@@ -332,3 +332,22 @@ def test_bench_configuration_sampled(pe):
         assert (gpu["makespan"] >= gpu["busy"].max(axis=0)).all() and (gpu["makespan"] >= ck.critical_path(w)).all()
     finally:
         g.close()
+
+
+def test_bounded_wait_reports_a_timeout_and_leaves_the_graph_usable(pe):
+    """The kernels' only wait (for the bulk copy that stages the graph) is bounded.  The self-test lets that wait
+    run out - a barrier that expects bytes no copy brings - and the host must read PE_ERR_TIMEOUT once, then
+    find the graph and the context in working order."""
+    w = wl.make_config(2)
+    K = 256
+    assign, order = wl.make_candidates(w, K=K)
+    g = pe.Graph(w)
+    try:
+        assert pe.pe_graph_poll_error(g.handle, 0) == pe.PE_OK
+        assert pe.pe_selftest_wait_timeout(g.handle, 0) == pe.PE_OK
+        assert pe.pe_graph_poll_error(g.handle, 0) == pe.PE_ERR_TIMEOUT
+        assert pe.pe_graph_poll_error(g.handle, 0) == pe.PE_OK          # reading clears it
+        gu.check(g, w, assign, order, label="after the self-test")
+        assert pe.pe_graph_poll_error(g.handle, 0) == pe.PE_OK
+    finally:
+        g.close()
