@@ -10,7 +10,10 @@ the three entry points working together on the device; it is not part of the eva
                pe_eval_batch scores them, the `elite` best feasible ones survive and the rest of
                the population is refilled with mutated copies of survivors (a few random rank
                swaps per list, a few reassigned operators per assignment);
-  result       pe_select_best of the last generation, and the best candidate seen.
+  result       the best candidate seen.
+
+`evolve` mutates lists and assignments directly; `evolve_keys` is the biased random-key variant for fixed
+assignments (a candidate is a vector of keys, its priority list their argsort).
 
 torch is used for the mutations (gather/scatter on the device) and for picking survivors;
 the scheduling arithmetic is all in the library's kernels.
@@ -60,4 +63,44 @@ def evolve(graph, assign, lists, generations=20, elite=0.125, swaps=2, reassign=
             i = torch.randint(0, V, (K,), device=dev, generator=gen)
             j = torch.randint(0, num_devices, (K,), device=dev, generator=gen).to(torch.uint8)
             assign[i, cols] = torch.where(mut, j, assign[i, cols])
+    return best
+
+
+def evolve_keys(graph, assign, generations=200, elite=0.1, mutants=0.2, bias=0.7, seed=0, reject_mask=0xFFFFFFFF,
+                flags=0):
+    """Biased random-key search over priority lists for fixed assignments (the random-key encoding of
+    sequencing problems: a candidate is a vector of keys in [0, 1), its priority list their argsort).
+    Each generation keeps the `elite` best, replaces the `mutants` worst by fresh random keys and fills
+    the rest by uniform crossover of an elite parent (each key taken with probability `bias`) with any
+    other candidate.  graph: binding.Graph; assign: cuda uint8 [V, K], column c is candidate c's assignment
+    throughout.  Returns dict(best_makespan, best_order [V], history)."""
+    import torch
+    V, K = assign.shape
+    dev = assign.device
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed)
+    n_el, n_mut = max(2, int(K * elite)), int(K * mutants)
+    big = torch.iinfo(torch.int32).max
+    mask_bits = int(np.uint32(reject_mask).view(np.int32))
+    keys = torch.rand((V, K), device=dev, generator=gen)
+    best = dict(best_makespan=big, history=[])
+    for _ in range(generations):
+        lists = torch.argsort(keys, dim=0).to(torch.int16).contiguous()
+        order, dstatus = graph.decode_priority(lists)
+        out = graph.eval_batch(assign, order, flags=flags, want_times=False)
+        bad = ((out["status"] & mask_bits) != 0) | (dstatus != 0)
+        score = torch.where(bad, torch.full_like(out["makespan"], big), out["makespan"])
+        top = torch.argsort(score, stable=True)[:n_el]
+        gbest = int(score[top[0]])
+        best["history"].append(gbest)
+        if gbest < best["best_makespan"]:
+            best.update(best_makespan=gbest, best_order=order[:, top[0]].clone(), best_column=int(top[0]))
+        pa = top[torch.randint(0, n_el, (K,), device=dev, generator=gen)]
+        pb = torch.randint(0, K, (K,), device=dev, generator=gen)
+        take = torch.rand((V, K), device=dev, generator=gen) < bias
+        child = torch.where(take, keys[:, pa], keys[:, pb])
+        child[:, :n_el] = keys[:, top]
+        if n_mut:
+            child[:, K - n_mut:] = torch.rand((V, n_mut), device=dev, generator=gen)
+        keys = child
     return best

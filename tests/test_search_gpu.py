@@ -35,5 +35,11 @@ def test_search_finds_the_pipeline_optimum_and_reports_what_the_oracle_computes(
         assert int(ref["makespan"][0]) == 72 and int(ref["status"][0]) == 0       # within the memory limit too
         dec, st = orc.decode(w, res["best_list"].cpu().numpy().view(np.uint16)[:, None])
         assert st[0] == 0 and np.array_equal(dec, o)
+        # the random-key variant (same assignment in every column) reaches the same optimum
+        rk = search.evolve_keys(g, assign, generations=80, seed=4)
+        assert rk["best_makespan"] == 72
+        o2 = rk["best_order"].cpu().numpy().view(np.uint16)[:, None]
+        ref2 = orc.evaluate(w, a, o2)
+        assert int(ref2["makespan"][0]) == 72 and int(ref2["status"][0]) == 0
     finally:
         g.close()
