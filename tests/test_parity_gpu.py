@@ -351,3 +351,37 @@ def test_bounded_wait_reports_a_timeout_and_leaves_the_graph_usable(pe):
         assert pe.pe_graph_poll_error(g.handle, 0) == pe.PE_OK
     finally:
         g.close()
+
+
+@pytest.mark.parametrize("V,D", [(256, 64), (1024, 8), (1024, 64), (4096, 8)])
+def test_other_sweep_points_at_full_size_sampled(pe, V, D):
+    """Sweep points at their full K (K * V = 2^30), i.e. in the launch shapes the benchmark times them in (ragged
+    shared-state blocks at V = 1024 / D = 8, slab mode of the warp kernel at V = 1024 / D = 64, register slots with
+    final rounds at V = 4096).  The batch repeats 8192 generated candidates; 256 sampled columns are compared
+    with the oracle in full, every column with its twin and with size-independent properties."""
+    import torch
+    from oracle import pe_oracle as orc
+    w = wl.make_config(5, V=V, D=D)
+    K, base = w.num_candidates, 8192
+    a0, o0 = wl.make_candidates(w, K=base)
+    assign = np.tile(a0, (1, K // base)); order = np.tile(o0, (1, K // base))
+    g = pe.Graph(w)
+    try:
+        a = torch.from_numpy(assign).cuda(); o = torch.from_numpy(gu.as_signed(order)).cuda()
+        out = g.eval_batch(a, o)
+        torch.cuda.synchronize()
+        rs = np.random.RandomState(V + D)
+        sample = np.sort(rs.choice(K, 256, replace=False))
+        st = torch.from_numpy(sample).cuda()
+        sub = {k: (v[st] if v.dim() == 1 else v[:, st]).cpu().numpy() for k, v in out.items()}
+        sub["status"] = sub["status"].view(np.uint32)
+        ref = orc.evaluate(w, np.ascontiguousarray(assign[:, sample]), np.ascontiguousarray(order[:, sample]),
+                           threads=gu.CPU_THREADS)
+        gu.compare(sub, ref, f"V={V} D={D} full size")
+        assert int(out["status"].abs().max()) == 0
+        assert bool((out["busy"].sum(dim=0) == int(w.dur.astype(np.int64).sum())).all())
+        assert bool((out["makespan"] == out["finish"].max(dim=0).values).all())
+        first = out["makespan"][:base]
+        assert bool((out["makespan"].view(K // base, base) == first).all())       # every repeat like its original
+    finally:
+        g.close()
