@@ -77,3 +77,30 @@ def test_which_kernels_offer_it(pe):
         assert pe.pe_workspace_bytes(g.handle, K, pe.PE_COMM_EXCLUSIVE) >= w.num_devices ** 2 * K * 4
     finally:
         g.close()
+
+
+def test_host_buffer_entry_point_with_exclusive_channels(pe):
+    import torch
+    from oracle import pe_oracle as orc
+    w = wl.make_config(4)
+    K = 3000
+    assign, order = wl.make_candidates(w, K=K)
+    flags = pe.PE_COMM_EXCLUSIVE
+    g = pe.Graph(w)
+    try:
+        h_a = torch.from_numpy(assign).pin_memory(); h_o = torch.from_numpy(gu.as_signed(order)).pin_memory()
+        d_a = torch.empty_like(h_a, device="cuda"); d_o = torch.empty_like(h_o, device="cuda")
+        d_out = g.alloc_outputs(K)
+        h_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in d_out.items()}
+        ws, ws_bytes = g.alloc_workspace(K, flags)
+        rc = pe.pe_eval_batch_host(g.handle, K, h_a.data_ptr(), h_o.data_ptr(), 2, flags,
+                                   pe.make_outputs(**{k: v.data_ptr() for k, v in h_out.items()}),
+                                   d_a.data_ptr(), d_o.data_ptr(),
+                                   pe.make_outputs(**{k: v.data_ptr() for k, v in d_out.items()}),
+                                   ws.data_ptr(), ws_bytes, torch.cuda.current_stream().cuda_stream)
+        assert rc == pe.PE_OK
+        res = {k: v.numpy() for k, v in h_out.items()}
+        res["status"] = res["status"].view(np.uint32)
+        gu.compare(res, orc.evaluate(w, assign, order, flags=orc.COMM_EXCLUSIVE, threads=gu.CPU_THREADS), "host call, exclusive")
+    finally:
+        g.close()
