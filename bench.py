@@ -46,7 +46,7 @@ KERNEL_OF_VARIANT = {"shared": "pe_eval_lane_kernel<STATE_SMEM=true>", "global":
 NCU_TRAFFIC = {
     # variant: (hash of csrc/ at capture time, DRAM bytes per operator-evaluation, captured workload)
     "global": ("0422252154d12689", 370.0, "random_layered_V16384_D64 at K = 32768 (half size), scaled by operator-evaluations"),
-    "warp": ("8711088e260103e9", 10.56, "random_layered_V16384_D64 at K = 4096, scaled by operator-evaluations"),
+    "warp": ("b3a5686239e56cfa", 10.59, "random_layered_V16384_D64 at K = 4096, scaled by operator-evaluations"),
 }
 
 

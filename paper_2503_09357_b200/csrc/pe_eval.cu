@@ -529,7 +529,9 @@ extern "C" int pe_eval_batch_host(pe_graph* g, int64_t K, const uint8_t* host_as
   // directions use separate DMA engines).  A chunk of Kc candidates lives in the staging buffers
   // as a dense [rows][Kc] block at element offset rows * first; the strided host side is handled
   // by 2-D copies.
-  int nchunks = K >= 8 * 4096 ? 8 : 1;
+  // (measured on the default workload: 16 chunks 6.1e9, 8 chunks 5.8e9, 4 chunks 5.3e9 operator-evaluations/s
+  // end to end - shorter chunks shorten the ramp before the first download and after the last upload)
+  int nchunks = K >= 16 * 4096 ? 16 : (K >= 8 * 4096 ? 8 : 1);
   const int64_t per = ((K + nchunks - 1) / nchunks + 255) / 256 * 256;
   nchunks = (int)((K + per - 1) / per);
   std::lock_guard<std::mutex> lock(g->host_mutex);
