@@ -38,7 +38,7 @@ DEFAULT_WORKLOAD = "random_layered_V16384_D64"   # the largest configuration: sw
 FALLBACK_HBM_GBS = 6650.0
 # the kernel each variant runs for graphs that have a compact encoding (all benchmark workloads do)
 KERNEL_OF_VARIANT = {"shared": "pe_eval_lane_kernel<STATE_SMEM=true>", "global": "pe_eval_lane_kernel<STATE_SMEM=false>",
-                     "warp": "pe_eval_warp2_kernel"}
+                     "warp": "pe_eval_warp2_kernel", "team": "pe_eval_team_kernel"}
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per operator-evaluation of the
 # evaluation kernel from an ncu capture, keyed by kernel variant, valid only for the kernel
@@ -51,7 +51,7 @@ NCU_TRAFFIC = {
 
 
 EVAL_SOURCES = ("pe_device.cuh", "pe_eval.cu", "pe_graph.cu", "pe_graph.h", "pe_kernel_lane.cuh", "pe_kernel_warp.cuh",
-                "pe_kernel_warp2.cuh", "pe_lane.cu", "pe_launch.h", "pe_warp2.cu")
+                "pe_kernel_warp2.cuh", "pe_kernel_team.cuh", "pe_lane.cu", "pe_launch.h", "pe_warp2.cu", "pe_team.cu")
 
 
 def kernel_source_hash():
@@ -256,7 +256,7 @@ def run_ours(args):
     V, D, K = w.num_ops, w.num_devices, (args.candidates or w.num_candidates)
     want_times = args.outputs == "full"
     flags = {"auto": pe.PE_VARIANT_AUTO, "global": pe.PE_VARIANT_GLOBAL, "shared": pe.PE_VARIANT_SHARED,
-             "warp": pe.PE_VARIANT_WARP}[args.variant]
+             "warp": pe.PE_VARIANT_WARP, "team": pe.PE_VARIANT_TEAM}[args.variant]
     obytes = 2 if V <= 65536 else 4
     odt = torch.int16 if obytes == 2 else torch.int32
 
@@ -447,7 +447,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default=DEFAULT_WORKLOAD)
     ap.add_argument("--outputs", choices=["full", "summary"], default="full")
-    ap.add_argument("--variant", choices=["auto", "global", "shared", "warp"], default="auto",
+    ap.add_argument("--variant", choices=["auto", "global", "shared", "warp", "team"], default="auto",
                     help="force a kernel variant (default: the library chooses)")
     ap.add_argument("--candidates", type=int, default=0, help="override K per GPU (default: the configuration's K)")
     ap.add_argument("--e2e-steps", type=int, default=3)

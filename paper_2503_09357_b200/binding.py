@@ -26,9 +26,10 @@ PE_ERR_SCRATCH_LIMIT = -9
 PE_NOALLOC_SCRATCH_BYTES = 64 << 20
 PE_ASSIGN_BY_POS, PE_TIMES_BY_OP, PE_COMM_EXCLUSIVE = 1, 2, 4
 PE_VARIANT_AUTO, PE_VARIANT_GLOBAL, PE_VARIANT_SHARED, PE_VARIANT_WARP = 0 << 8, 1 << 8, 2 << 8, 3 << 8
+PE_VARIANT_TEAM = 4 << 8
 PE_VARIANT_MASK = 15 << 8
 PE_STATUS_ASSIGN_RANGE, PE_STATUS_ORDER_INVALID, PE_STATUS_MEM_EXCEEDED, PE_STATUS_NO_CHANNEL = 1, 2, 4, 8
-VARIANT_NAMES = {PE_VARIANT_GLOBAL: "global", PE_VARIANT_SHARED: "shared", PE_VARIANT_WARP: "warp"}
+VARIANT_NAMES = {PE_VARIANT_GLOBAL: "global", PE_VARIANT_SHARED: "shared", PE_VARIANT_WARP: "warp", PE_VARIANT_TEAM: "team"}
 
 _P = ctypes.c_void_p
 

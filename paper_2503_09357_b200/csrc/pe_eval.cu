@@ -15,6 +15,7 @@
 #include "pe_graph.h"
 #include "pe_kernel_warp.cuh"
 #include "pe_launch.h"
+#include <cstdlib>
 
 namespace pe {
 
@@ -305,6 +306,43 @@ static bool plan_warp(const pe_graph* g, int64_t K, uint32_t flags, bool allow_c
   return true;
 }
 
+// TEAM: one block per candidate; plan.threads / 32 warps share the candidate's windows.  With K a multiple of 4
+// (the transpositions move 32-bit words) the inputs and the times go through candidate-major staging copies
+// in the workspace, a chunk of candidates at a time; a chunk is sixteen times what the GPU holds at once.
+static bool plan_team(const pe_graph* g, int64_t K, bool allow_compact, Plan* p) {
+  if (!g->narrow_ok || !allow_compact || g->max_indeg > 3 || g->time_bound >= (int64_t)1 << 23) return false;
+  const size_t smem = round_up((size_t)4 * (g->V + 1) + (size_t)4 * (5 * g->D + 2), 16);
+  if (smem > g->smem_optin) return false;
+  int nw = 6;
+  if (const char* e = std::getenv("PE_TEAM_WARPS")) nw = std::atoi(e);
+  if (nw != 2 && nw != 4 && nw != 6) return false;
+  p->variant = PE_VARIANT_TEAM;
+  p->threads = 32 * nw;
+  p->smem = smem;
+  p->graph_smem = false;
+  p->workspace = 0;
+  p->ws_x_off = 0;
+  p->compact = true;
+  p->staged = K >= 64 && K % 4 == 0 && !std::getenv("PE_TEAM_DIRECT");
+  if (p->staged) {
+    size_t per_sm = (g->smem_per_sm ? g->smem_per_sm : g->smem_optin) / (smem + 1024);
+    if (per_sm < 1) per_sm = 1;
+    if (per_sm * p->threads > 2048) per_sm = 2048 / p->threads;
+    int64_t chunk = (int64_t)per_sm * g->sm_count * 16 / 4 * 4;
+    if (chunk > K) chunk = K;
+    p->team_chunk = chunk;
+    p->team_vp = ((int64_t)g->V + 63) / 64 * 64;
+    const size_t cells = (size_t)chunk * (size_t)p->team_vp;
+    size_t at = 0;
+    p->team_off_order = at;  at = round_up(at + cells * 2, 256);
+    p->team_off_assign = at; at = round_up(at + cells, 256);
+    p->team_off_start = at;  at = round_up(at + cells * 4, 256);
+    p->team_off_finish = at; at = round_up(at + cells * 4, 256);
+    p->workspace = at;
+  }
+  return true;
+}
+
 static bool plan_global(const pe_graph* g, int64_t K, uint32_t flags, bool allow_compact, Plan* p) {
   p->compact = false;
   const bool exclusive = (flags & PE_COMM_EXCLUSIVE) != 0;   // only the generic kernel sequences transfers per channel
@@ -389,6 +427,7 @@ static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, bool allow_co
     case PE_VARIANT_GLOBAL: return plan_global(g, K, flags, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
     case PE_VARIANT_SHARED: return plan_shared(g, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
     case PE_VARIANT_WARP: return plan_warp(g, K, flags, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+    case PE_VARIANT_TEAM: return plan_team(g, K, allow_compact, p) ? PE_OK : PE_ERR_UNSUPPORTED;
     default: return PE_ERR_UNSUPPORTED;
   }
 }
@@ -398,13 +437,21 @@ template <typename OrderT, bool BY_POS>
 static int launch_typed(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* assign, const void* order,
                         uint32_t flags, const pe_outputs& out, void* workspace, cudaStream_t stream) {
   const PeGraphView view = pe_view(g);
-  const int per_block = p.variant == PE_VARIANT_WARP ? p.threads / 32 : p.threads;  // candidates per block
+  const int per_block = p.variant == PE_VARIANT_TEAM ? 1 : (p.variant == PE_VARIANT_WARP ? p.threads / 32 : p.threads);  // candidates per block
   const unsigned grid = (unsigned)((K + per_block - 1) / per_block);
   const OrderT* ord = static_cast<const OrderT*>(order);
   if (p.compact) {
     if (sizeof(OrderT) != 2) return PE_ERR_INVALID_ARG;
     const uint16_t* ord16 = static_cast<const uint16_t*>(order);
     uint32_t* gstate = static_cast<uint32_t*>(workspace);
+    if (p.variant == PE_VARIANT_TEAM) {
+      if (p.staged && (((uintptr_t)assign | (uintptr_t)order) & 3u)) return PE_ERR_INVALID_ARG;   // word-wise transpositions
+      int64_t n = 0;
+      const int rc = launch_team(g, p, BY_POS, K, assign, ord16, flags, out, workspace, stream, &n);
+      if (rc != PE_OK) return rc;
+      g_launches.fetch_add(n, std::memory_order_relaxed);
+      return cudaGetLastError() == cudaSuccess ? PE_OK : PE_ERR_CUDA;
+    }
     const int rc = p.variant == PE_VARIANT_WARP ? launch_warp2(g, p, BY_POS, K, assign, ord16, flags, out, grid, stream)
                                                 : launch_lane(g, p, BY_POS, K, assign, ord16, flags, out, gstate, grid, stream);
     if (rc != PE_OK) return rc;

@@ -221,6 +221,7 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
   if (ok) {
     g->sm_count = prop.multiProcessorCount;
     g->smem_optin = prop.sharedMemPerBlockOptin;
+    g->smem_per_sm = prop.sharedMemPerMultiprocessor;
     ok = cudaMalloc((void**)&g->d_blob, lay.bytes) == cudaSuccess &&
          cudaMalloc((void**)&g->d_error, 256) == cudaSuccess &&
          cudaMemcpy(g->d_blob, blob.data(), lay.bytes, cudaMemcpyHostToDevice) == cudaSuccess &&

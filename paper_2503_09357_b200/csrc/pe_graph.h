@@ -96,6 +96,7 @@ struct pe_graph {
   std::mutex host_mutex;
   int sm_count;
   size_t smem_optin;   // max dynamic shared memory per block
+  size_t smem_per_sm;  // shared memory of an SM
 };
 
 inline PeGraphView pe_view(const pe_graph* g) {

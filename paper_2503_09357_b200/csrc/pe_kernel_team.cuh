@@ -1,0 +1,386 @@
+// Variant TEAM over the compact graph encoding: one block per candidate, NW warps that take the
+// windows of 32 consecutive positions of the priority order in turn, per-operator state in shared
+// memory.
+//
+// When a candidate's state (4 bytes per operator) is so large that only a handful fit on an SM, a
+// single warp per candidate leaves the SM idle: a window then costs the latency of everything it
+// does, one thing after the other.  Most of that work does not depend on any start or end time:
+// which operator sits at a position, its record, the machines of its predecessors and hence the
+// delay of each incoming edge (Eqs. 9, 11-13), whether a predecessor sits in the same window, which
+// operator precedes it on its machine inside the window (Eqs. 7-8), the memory levels (Eqs. 16-19).
+// Only the recurrence itself, s_i = max(ready, free_j), e_i = s_i + D^o_i (Eqs. 3, 7-8, 11-13), has
+// to follow the order.  So the block works as a pipeline:
+//   * an initial pass writes every operator's position in the order and its machine into the state
+//     word ("pending": position << 8 | machine), so that later nobody has to wait to learn where a
+//     predecessor sits;
+//   * warp w prepares windows w, w + NW, ... on its own: it reads the order entries and operator
+//     records (prefetched), classifies the incoming edges into sources inside the window (lane,
+//     delay) and sources before it (state address, delay), and finds the machine's previous
+//     operator in the window;
+//   * a baton (a named barrier between two warps) goes from window to window.  The warp that holds
+//     it gathers the end times of the sources before the window (final by then), relaxes the window
+//     with shuffles until nothing changes, publishes end << 8 | machine and passes the baton on.
+//     Only this part is serial, and it touches nothing but shared memory and registers;
+//   * the memory levels follow each machine's sequence, not the times: they have their own, much
+//     shorter, baton, and run ahead of the times.
+// State word: pending = 0x80000000 | position << 8 | machine (position 0xFFFF = not in the order);
+// final = end << 8 | machine, end < 2^23.  Row V is the sentinel the compact encoding's empty edge
+// slots point at (final, end 0, machine 0).
+//
+// The kernel serves graphs in which no operator has more than three incoming edges (the inline
+// slots of the compact record are then all there is).
+#pragma once
+#include "pe_device.cuh"
+#include "pe_kernel_lane.cuh"
+
+namespace pe {
+
+constexpr uint32_t kTeamPending = 0x80000000u;
+constexpr int64_t kTeamTimeLimit = (int64_t)1 << 23;   // end times must stay below this
+
+// Named barriers: `count` threads in all; the warps that call named_arrive do not wait.
+__device__ __forceinline__ void named_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void named_arrive(int id, int count) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+// Element (row, c) of an input or output array sits at row * row_stride + c * cand_stride: (K, 1) for
+// the candidate-interleaved arrays of the interface, (1, rows) for candidate-major staging copies.
+struct TeamStrides {
+  size_t in_row, in_cand;     // assign, order
+  size_t out_row, out_cand;   // start, finish
+};
+
+template <int NW, bool BY_POS, int CLS, bool TIMES, bool STAGED>
+__global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, const uint8_t* __restrict__ nblob,
+                                                               int64_t K, const uint8_t* __restrict__ assign,
+                                                               const uint16_t* __restrict__ order, pe_outputs out,
+                                                               uint32_t flags, TeamStrides sd) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  static_assert(2 * NW + 1 <= 16, "two named barriers per warp, barrier 0 is the block's");
+  constexpr uint32_t FULL = 0xFFFFFFFFu;
+  constexpr bool TWO_CLASS = CLS == 2;
+  constexpr bool NEED_CLS = CLS != 0;
+  constexpr int NT = NW * 32;
+  constexpr int32_t kNever = -(1 << 29);   // delay of an empty slot: never wins the maximum
+  const int tid = threadIdx.x;
+  const int lane = tid & 31;
+  const int warp = tid >> 5;
+  const int D = g.D, V = g.V;
+  const NarrowPtrs gp = narrow_ptrs(nblob, g);
+  const int64_t c = blockIdx.x;
+  const uint32_t vmax = (uint32_t)(V - 1), dmax = (uint32_t)(D - 1);
+
+  uint32_t* state = reinterpret_cast<uint32_t*>(smem_raw);   // [V + 1]
+  int32_t* free_at = reinterpret_cast<int32_t*>(state + V + 1);
+  int32_t* lvl = free_at + D;
+  int32_t* peak = lvl + D;
+  int32_t* busy = peak + D;
+  int32_t* wsum = busy + D;
+  int32_t* red = wsum + D;   // [0] makespan, [1] status
+
+  const uint16_t* order_col = order + (size_t)c * sd.in_cand;
+  const uint8_t* assign_col = assign + (size_t)c * sd.in_cand;
+  uint32_t st = 0;
+  uint32_t order_max = 0, dev_max = 0;
+
+  // ---- initial pass: machine and position of every operator ----
+  for (int idx = tid; idx < 5 * D + 2; idx += NT) free_at[idx] = 0;
+  if (tid == 0) state[V] = 0u;
+  constexpr int kBatch = 8;   // loads in flight per thread
+  if constexpr (STAGED) {
+    // candidate-major staging copies: the candidate's machine ids and order entries are contiguous
+    // (rows padded with zeros to a multiple of 64 entries), four entries per load
+    const uint32_t* a4 = reinterpret_cast<const uint32_t*>(assign_col);
+    const uint2* o4 = reinterpret_cast<const uint2*>(order_col);
+    const int nq = (V + 3) >> 2;
+    for (int b = tid; b < nq; b += NT * kBatch) {
+      uint32_t x[kBatch];
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q) {
+        const int v4 = b + q * NT;
+        x[q] = (!BY_POS && v4 < nq) ? a4[v4] : 0u;
+      }
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q) {
+        const int v4 = b + q * NT;
+        if (v4 < nq) {
+#pragma unroll
+          for (int h = 0; h < 4; ++h)
+            if (4 * v4 + h < V) state[4 * v4 + h] = kTeamPending | 0xFFFF00u | ((x[q] >> (8 * h)) & 0xFFu);
+        }
+      }
+    }
+    __syncthreads();
+    for (int b = tid; b < nq; b += NT * kBatch) {
+      uint2 o[kBatch];
+      uint32_t a[kBatch];
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q) {
+        const int v4 = b + q * NT;
+        o[q] = v4 < nq ? o4[v4] : make_uint2(0xFFFFFFFFu, 0xFFFFFFFFu);
+        a[q] = (BY_POS && v4 < nq) ? a4[v4] : 0u;
+      }
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q) {
+        const int v4 = b + q * NT;
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+          const int k = 4 * v4 + h;
+          const uint32_t oe = ((h < 2 ? o[q].x : o[q].y) >> (16 * (h & 1))) & 0xFFFFu;
+          const uint32_t ae = (a[q] >> (8 * h)) & 0xFFu;
+          if (v4 < nq && k < V && oe <= vmax) {
+            if (BY_POS) {
+              dev_max = max(dev_max, ae);
+              state[oe] = kTeamPending | ((uint32_t)k << 8) | ae;
+            } else {
+              state[oe] = kTeamPending | ((uint32_t)k << 8) | (state[oe] & 0xFFu);
+            }
+          }
+        }
+      }
+    }
+    __syncthreads();
+  } else {
+  for (int b = tid; b < V; b += NT * kBatch) {
+    uint32_t x[kBatch];
+#pragma unroll
+    for (int q = 0; q < kBatch; ++q) {
+      const int i = b + q * NT;
+      x[q] = (!BY_POS && i < V) ? (uint32_t)assign_col[(size_t)i * sd.in_row] : 0u;
+    }
+#pragma unroll
+    for (int q = 0; q < kBatch; ++q) {
+      const int i = b + q * NT;
+      if (i < V) state[i] = kTeamPending | 0xFFFF00u | x[q];
+    }
+  }
+  __syncthreads();
+  for (int b = tid; b < V; b += NT * kBatch) {
+    uint32_t o[kBatch], a[kBatch];
+#pragma unroll
+    for (int q = 0; q < kBatch; ++q) {
+      const int k = b + q * NT;
+      o[q] = k < V ? (uint32_t)order_col[(size_t)k * sd.in_row] : 0xFFFFFFFFu;
+      a[q] = (BY_POS && k < V) ? (uint32_t)assign_col[(size_t)k * sd.in_row] : 0u;
+    }
+#pragma unroll
+    for (int q = 0; q < kBatch; ++q) {
+      const int k = b + q * NT;
+      if (o[q] <= vmax) {
+        if (BY_POS) {
+          dev_max = max(dev_max, a[q]);
+          state[o[q]] = kTeamPending | ((uint32_t)k << 8) | a[q];
+        } else {
+          state[o[q]] = kTeamPending | ((uint32_t)k << 8) | (state[o[q]] & 0xFFu);
+        }
+      }
+    }
+  }
+  __syncthreads();
+  }
+
+  const bool by_op_times = (flags & PE_TIMES_BY_OP) != 0;
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  const int nwin = (V + 31) >> 5;
+  const int next_warp = (warp + 1) % NW;
+  int32_t z = 0;
+  int32_t* start_col = TIMES ? out.start + (size_t)c * sd.out_cand : nullptr;
+  int32_t* finish_col = TIMES ? out.finish + (size_t)c * sd.out_cand : nullptr;
+
+  auto load_order = [&](int win) -> uint32_t {
+    const int k = win * 32 + lane;
+    return k < V ? (uint32_t)order_col[(size_t)k * sd.in_row] : 0u;
+  };
+  // order entries two of this warp's windows ahead, operator records one ahead
+  uint32_t o_cur = load_order(warp), o_nxt = load_order(warp + NW);
+  uint4 rec_nxt = __ldg(gp.ops + min(o_cur, vmax));
+
+  for (int win = warp; win < nwin; win += NW) {
+    const int base = win * 32;
+    const int k = base + lane;
+    const bool act = k < V;
+    const uint32_t iu = o_cur;
+    const uint4 rec = rec_nxt;
+    o_cur = o_nxt;
+    o_nxt = load_order(win + 2 * NW);
+    rec_nxt = __ldg(gp.ops + min(o_cur, vmax));
+
+    // ---- set-up: nothing here depends on a time ----
+    if (act) order_max = max(order_max, iu);
+    const uint32_t i = act ? min(iu, vmax) : (uint32_t)V;
+    const uint32_t own = state[i];
+    if (act && (own >> 8) != ((kTeamPending >> 8) | (uint32_t)k)) st |= PE_STATUS_ORDER_INVALID;  // repeated operator
+    const uint32_t jr = own & 0xFFu;
+    if (!BY_POS && act) dev_max = max(dev_max, jr);
+    const uint32_t j = min(jr, dmax);
+    const int indeg = (int)(rec.y >> 24);
+    const int32_t dur = act ? (int32_t)(rec.y & 0xFFFFu) : 0;
+    const int32_t dA = act ? (int32_t)(rec.y << 8) >> 24 : 0;
+
+    // previous / last operator of the same machine inside the window (Eqs. 7-8)
+    const uint32_t same_dev = __match_any_sync(FULL, act ? j : (0x100u | lane));
+    const uint32_t below = same_dev & lt_mask;
+    const int prev = below ? 31 - __clz(below) : -1;
+    const bool last_on_dev = (same_dev >> lane) == 1u;
+
+    // incoming edges: edge q owns slot q.  A source inside the window becomes (lane, delay) for the
+    // relaxation; any other becomes (state address, delay) for the gather under the baton.  The unused
+    // half of a slot is neutral: lane = own lane with delay kNever, address = sentinel with delay kNever.
+    const uint32_t none = (uint32_t)V;
+    uint32_t a0 = none, a1 = none, a2 = none;
+    int32_t g0 = kNever, g1 = kNever, g2 = kNever;
+    int l0 = lane, l1 = lane, l2 = lane;
+    int32_t d0 = kNever, d1 = kNever, d2 = kNever;
+    uint32_t depmask = 0;
+    auto delay_of = [&](uint32_t lo, uint32_t hi, uint32_t w) -> uint32_t {
+      const uint32_t xp = w & 0xFFu;
+      uint32_t delay = lo >> 16;
+      if (NEED_CLS) {
+        const uint32_t cl = gp.cls[min(xp, dmax) * D + j];
+        if (TWO_CLASS) delay = cl == 1u ? hi : delay;
+        if (cl == 0xFFu) {
+          delay = 0;
+          if ((lo & 0xFFFFu) != none && xp != j) st |= PE_STATUS_NO_CHANNEL;
+        }
+      }
+      return xp != j ? delay : 0u;
+    };
+    auto classify = [&](uint32_t lo, uint32_t hi, uint32_t& addr, int32_t& gdel, int& lsl, int32_t& ldel) {
+      const uint32_t p = lo & 0xFFFFu;
+      const uint32_t w = state[p];
+      const int32_t dly = (int32_t)delay_of(lo, hi, w);
+      const uint32_t pos = (w >> 8) & 0xFFFFu;
+      if ((w & kTeamPending) && pos >= (uint32_t)base) {
+        if (pos < (uint32_t)k) {
+          lsl = (int)(pos - (uint32_t)base);
+          ldel = dly;
+          depmask |= 1u << lsl;
+        } else {
+          st |= PE_STATUS_ORDER_INVALID;   // a predecessor that is not before this operator
+        }
+      } else {
+        addr = p;   // final already, or in an earlier window: final by the time the baton arrives
+        gdel = dly;
+      }
+    };
+    if (act) {
+      classify(rec.z, rec.w, a0, g0, l0, d0);
+      if (TWO_CLASS) {
+        const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
+        if (indeg > 1) { const uint2 e1 = __ldg(ed + 1); classify(e1.x, e1.y, a1, g1, l1, d1); }
+        if (indeg > 2) { const uint2 e2 = __ldg(ed + 2); classify(e2.x, e2.y, a2, g2, l2, d2); }
+      } else {
+        classify(rec.w, 0u, a1, g1, l1, d1);
+        classify(rec.x, 0u, a2, g2, l2, d2);
+      }
+    }
+    int lp = lane;
+    int32_t dp = kNever;
+    if (act && prev >= 0) { lp = prev; dp = 0; depmask |= 1u << prev; }
+    // Depth of the window: peel off, round by round, the lanes whose sources are all peeled.  After r
+    // rounds of relaxation every lane of depth <= r holds its final value, so the number of rounds the
+    // baton has to wait for is known before it arrives and the loop under it needs no vote.
+    int nrounds = 0;
+    {
+      bool fin = depmask == 0;
+      uint32_t done = __ballot_sync(FULL, fin);
+      while (done != FULL) {
+        fin = fin || (depmask & ~done) == 0;
+        done = __ballot_sync(FULL, fin);
+        ++nrounds;
+      }
+    }
+    // e_l = max(r_base, max_q(e_src(q) + delay_q)) + D^o (Eqs. 3, 7-8, 11-13) with D^o folded into the delays
+    d0 += dur; d1 += dur; d2 += dur; dp += dur;
+
+    // ---- memory levels (Eqs. 17-19): prefix sums of A along each machine's lanes, then the machine's
+    // level before the window, under the ledger baton ----
+    int32_t lv = dA;
+    {
+      uint32_t m = below;
+      while (__any_sync(FULL, m != 0)) {
+        const int src = m ? __ffs(m) - 1 : lane;
+        const int32_t a_src = __shfl_sync(FULL, dA, src);
+        if (m) { lv += a_src; m &= m - 1; }
+      }
+    }
+    if (act) {
+      atomicAdd(&busy[j], dur);
+      if (gp.weight) atomicAdd(&wsum[j], gp.weight[i]);
+    }
+    if (win > 0) named_sync(1 + NW + warp, 64);
+    if (act) {
+      lv += lvl[j];
+      atomicMax(&peak[j], lv);
+    }
+    __syncwarp();
+    if (act && last_on_dev) lvl[j] = lv;
+    __syncwarp();
+    if (win + 1 < nwin) named_arrive(1 + NW + next_warp, 64);
+
+    // ---- times, under the baton: every earlier window is final ----
+    if (win > 0) named_sync(1 + warp, 64);
+    const uint32_t w0 = state[a0], w1 = state[a1], w2 = state[a2];
+    int32_t r_base = (act && prev < 0) ? free_at[j] : 0;
+    r_base = max(r_base, (int32_t)(w0 >> 8) + g0);
+    r_base = max(r_base, (int32_t)(w1 >> 8) + g1);
+    r_base = max(r_base, (int32_t)(w2 >> 8) + g2);
+    const int32_t b_end = r_base + dur;
+    int32_t e = b_end;
+    // every dependence points to a lower lane, so the values rise monotonically to the window's
+    // longest-path solution, which they reach after `nrounds` rounds
+    for (int it = 0; it < nrounds; ++it) {
+      const int32_t t0 = __shfl_sync(FULL, e, l0) + d0;
+      const int32_t t1 = __shfl_sync(FULL, e, l1) + d1;
+      const int32_t t2 = __shfl_sync(FULL, e, l2) + d2;
+      const int32_t t3 = __shfl_sync(FULL, e, lp) + dp;
+      e = max(max(b_end, t0), max(max(t1, t2), t3));
+    }
+    if (act) {
+      state[i] = ((uint32_t)e << 8) | j;
+      if (last_on_dev) free_at[j] = e;
+    }
+    __syncwarp();
+    if (win + 1 < nwin) named_arrive(1 + next_warp, 64);
+
+    // ---- after the baton has gone: outputs ----
+    z = max(z, e);
+    if (TIMES && act) {
+      const size_t at = (size_t)(by_op_times ? i : (uint32_t)k) * sd.out_row;
+      start_col[at] = e - dur;
+      finish_col[at] = e;
+    }
+  }
+
+  if (order_max > vmax) st |= PE_STATUS_ORDER_INVALID;
+  if (dev_max > dmax) st |= PE_STATUS_ASSIGN_RANGE;
+  for (int off = 16; off > 0; off >>= 1) {
+    z = max(z, __shfl_xor_sync(FULL, z, off));
+    st |= __shfl_xor_sync(FULL, st, off);
+  }
+  if (lane == 0) {
+    atomicMax(&red[0], z);
+    atomicOr(reinterpret_cast<uint32_t*>(&red[1]), st);
+  }
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t over = 0;
+    for (int j = lane; j < D; j += 32) {
+      const int32_t pk = peak[j] + (gp.weight ? wsum[j] : 0);   // the weights are resident from the start (Eq. 16)
+      if (pk > gp.cap[j]) over = 1;
+      if (out.busy) out.busy[(size_t)j * (size_t)K + c] = busy[j];
+      if (out.peak_mem) out.peak_mem[(size_t)j * (size_t)K + c] = pk;
+    }
+    uint32_t stf = (uint32_t)red[1];
+    if (__any_sync(FULL, over != 0)) stf |= PE_STATUS_MEM_EXCEEDED;
+    if (lane == 0) {
+      if (out.makespan) out.makespan[c] = red[0];
+      if (out.status) out.status[c] = stf;
+    }
+  }
+}
+
+}  // namespace pe

@@ -21,6 +21,11 @@ struct Plan {
   bool compact = false;   // SHARED / GLOBAL / WARP: the compact-graph kernels
   bool exclusive = false; // SHARED (compact): PE_COMM_EXCLUSIVE, one more word per machine pair and candidate
   bool slab = false;      // WARP (compact): order entries and times go through shared tiles, a slab at a time
+  // TEAM: inputs and times go through candidate-major staging copies in the workspace, a chunk of candidates at a time
+  bool staged = false;
+  int64_t team_chunk = 0;   // candidates per chunk (multiple of 4)
+  int64_t team_vp = 0;      // row length of the staging copies: V rounded up to a multiple of 64
+  size_t team_off_order = 0, team_off_assign = 0, team_off_start = 0, team_off_finish = 0;   // offsets in the workspace
 };
 
 template <typename Kern>
@@ -35,5 +40,10 @@ int launch_lane(const pe_graph* g, const Plan& p, bool by_pos, int64_t K, const 
 // pe_eval_warp2_kernel (plan variant WARP over the compact encoding).
 int launch_warp2(const pe_graph* g, const Plan& p, bool by_pos, int64_t K, const uint8_t* assign, const uint16_t* order,
                  uint32_t flags, const pe_outputs& out, unsigned grid, cudaStream_t stream);
+
+// pe_eval_team_kernel (plan variant TEAM: one block of plan.threads / 32 warps per candidate).
+// Adds the number of kernels it launched to *launches.
+int launch_team(const pe_graph* g, const Plan& p, bool by_pos, int64_t K, const uint8_t* assign, const uint16_t* order,
+                uint32_t flags, const pe_outputs& out, void* workspace, cudaStream_t stream, int64_t* launches);
 
 }  // namespace pe

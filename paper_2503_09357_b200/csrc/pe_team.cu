@@ -1,0 +1,110 @@
+// Instantiations and launcher of pe_eval_team_kernel, with the staging transpositions around it.
+#include "pe_kernel_team.cuh"
+#include "pe_launch.h"
+#include "pe_transpose.cuh"
+
+namespace pe {
+
+namespace {
+
+struct TeamCall {
+  const pe_graph* g;
+  const Plan* p;
+  int64_t K;        // row pitch of the interface arrays
+  int64_t kc;       // candidates of this launch
+  const uint8_t* assign;
+  const uint16_t* order;
+  uint32_t flags;
+  pe_outputs out;
+  TeamStrides sd;
+  cudaStream_t stream;
+};
+
+template <int NW, bool BY_POS, int CLS>
+int launch3(const TeamCall& t) {
+  auto go = [&](auto kern) -> int {
+    if (!set_smem(kern, t.p->smem)) return PE_ERR_CUDA;
+    kern<<<(unsigned)t.kc, NW * 32, t.p->smem, t.stream>>>(t.g->nview, t.g->d_nblob, t.K, t.assign, t.order, t.out, t.flags,
+                                                            t.sd);
+    return PE_OK;
+  };
+  if (t.p->staged)
+    return t.out.start ? go(pe_eval_team_kernel<NW, BY_POS, CLS, true, true>)
+                       : go(pe_eval_team_kernel<NW, BY_POS, CLS, false, true>);
+  return t.out.start ? go(pe_eval_team_kernel<NW, BY_POS, CLS, true, false>)
+                     : go(pe_eval_team_kernel<NW, BY_POS, CLS, false, false>);
+}
+
+template <int NW, bool BY_POS>
+int launch2(const TeamCall& t) {
+  const int cls = t.g->nview.L == 2 ? 2 : (t.g->nview.need_cls ? 1 : 0);
+  if (cls == 2) return launch3<NW, BY_POS, 2>(t);
+  if (cls == 1) return launch3<NW, BY_POS, 1>(t);
+  return launch3<NW, BY_POS, 0>(t);
+}
+
+template <bool BY_POS>
+int launch1(const TeamCall& t) {
+  switch (t.p->threads / 32) {
+    case 2: return launch2<2, BY_POS>(t);
+    case 4: return launch2<4, BY_POS>(t);
+    case 6: return launch2<6, BY_POS>(t);
+    default: return PE_ERR_UNSUPPORTED;
+  }
+}
+
+// out[C][out_ld] = transposed in[R][in_ld] (element size S)
+template <int S>
+void transpose(const void* in, void* out, int64_t R, int64_t C, int64_t in_ld, int64_t out_ld, cudaStream_t stream) {
+  constexpr int TR = 32 * (4 / S);
+  const dim3 grid((unsigned)((C + TR - 1) / TR), (unsigned)((R + TR - 1) / TR));
+  pe_transpose_kernel<S><<<grid, 256, 0, stream>>>(static_cast<const uint8_t*>(in), static_cast<uint8_t*>(out), R, C, in_ld,
+                                                   out_ld);
+}
+
+}  // namespace
+
+int launch_team(const pe_graph* g, const Plan& p, bool by_pos, int64_t K, const uint8_t* assign, const uint16_t* order,
+                uint32_t flags, const pe_outputs& out, void* workspace, cudaStream_t stream, int64_t* launches) {
+  TeamCall t;
+  t.g = g; t.p = &p; t.K = K; t.flags = flags; t.stream = stream;
+  if (!p.staged) {
+    t.kc = K; t.assign = assign; t.order = order; t.out = out;
+    t.sd.in_row = (size_t)K; t.sd.in_cand = 1; t.sd.out_row = (size_t)K; t.sd.out_cand = 1;
+    *launches += 1;
+    return by_pos ? launch1<true>(t) : launch1<false>(t);
+  }
+  // staged: chunks of candidates go through candidate-major copies in the workspace
+  const int64_t V = g->V, D = g->D, Vp = p.team_vp;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  uint16_t* ord_t = reinterpret_cast<uint16_t*>(ws + p.team_off_order);
+  uint8_t* asg_t = ws + p.team_off_assign;
+  int32_t* start_t = reinterpret_cast<int32_t*>(ws + p.team_off_start);
+  int32_t* finish_t = reinterpret_cast<int32_t*>(ws + p.team_off_finish);
+  const bool times = out.start != nullptr;
+  for (int64_t c0 = 0; c0 < K; c0 += p.team_chunk) {
+    const int64_t kc = K - c0 < p.team_chunk ? K - c0 : p.team_chunk;
+    transpose<2>(order + c0, ord_t, V, kc, K, Vp, stream);
+    transpose<1>(assign + c0, asg_t, V, kc, K, Vp, stream);
+    t.kc = kc; t.assign = asg_t; t.order = ord_t;
+    t.out.start = times ? start_t : nullptr;
+    t.out.finish = times ? finish_t : nullptr;
+    t.out.makespan = out.makespan ? out.makespan + c0 : nullptr;
+    t.out.status = out.status ? out.status + c0 : nullptr;
+    t.out.busy = out.busy ? out.busy + c0 : nullptr;
+    t.out.peak_mem = out.peak_mem ? out.peak_mem + c0 : nullptr;
+    t.sd.in_row = 1; t.sd.in_cand = (size_t)Vp; t.sd.out_row = 1; t.sd.out_cand = (size_t)Vp;
+    const int rc = by_pos ? launch1<true>(t) : launch1<false>(t);
+    if (rc != PE_OK) return rc;
+    *launches += 3;
+    if (times) {
+      transpose<4>(start_t, out.start + c0, kc, V, Vp, K, stream);
+      transpose<4>(finish_t, out.finish + c0, kc, V, Vp, K, stream);
+      *launches += 2;
+    }
+  }
+  (void)D;
+  return PE_OK;
+}
+
+}  // namespace pe

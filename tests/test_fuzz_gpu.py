@@ -51,7 +51,7 @@ def test_random_problems_match_the_oracle_in_every_variant(seed):
     g = pe.Graph(w)
     try:
         for name, bit in (("auto", 0), ("global", pe.PE_VARIANT_GLOBAL), ("shared", pe.PE_VARIANT_SHARED),
-                          ("warp", pe.PE_VARIANT_WARP), ("exclusive", pe.PE_COMM_EXCLUSIVE),
+                          ("warp", pe.PE_VARIANT_WARP), ("team", pe.PE_VARIANT_TEAM), ("exclusive", pe.PE_COMM_EXCLUSIVE),
                           ("exclusive shared", pe.PE_COMM_EXCLUSIVE | pe.PE_VARIANT_SHARED),
                           ("exclusive global", pe.PE_COMM_EXCLUSIVE | pe.PE_VARIANT_GLOBAL)):
             if pe.pe_eval_variant(g.handle, K, base | bit) < 0:

@@ -42,7 +42,8 @@ def test_evaluation_at_the_largest_sizes(pe, V):
     g = pe.Graph(w)
     try:
         seen = set()
-        for name, bit in (("auto", 0), ("global", pe.PE_VARIANT_GLOBAL), ("warp", pe.PE_VARIANT_WARP)):
+        for name, bit in (("auto", 0), ("global", pe.PE_VARIANT_GLOBAL), ("warp", pe.PE_VARIANT_WARP),
+                          ("team", pe.PE_VARIANT_TEAM)):
             if pe.pe_eval_variant(g.handle, K, bit) < 0:
                 continue
             gu.check(g, w, assign, order, flags=bit, label=f"V={V} {name}")

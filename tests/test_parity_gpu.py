@@ -20,7 +20,8 @@ def pe():
 
 def variants_for(pe, graph, K, base_flags=0):
     out = [("auto", base_flags)]
-    for name, bit in (("global", pe.PE_VARIANT_GLOBAL), ("shared", pe.PE_VARIANT_SHARED), ("warp", pe.PE_VARIANT_WARP)):
+    for name, bit in (("global", pe.PE_VARIANT_GLOBAL), ("shared", pe.PE_VARIANT_SHARED), ("warp", pe.PE_VARIANT_WARP),
+                      ("team", pe.PE_VARIANT_TEAM)):
         if pe.pe_eval_variant(graph.handle, K, base_flags | bit) >= 0:
             out.append((name, base_flags | bit))
     return out
@@ -130,6 +131,11 @@ def test_u32_orders(pe):
     g = pe.Graph(w)
     try:
         for name, flags in variants_for(pe, g, K):
+            if name == "team":                              # 16-bit orders only: refused, not mis-evaluated
+                with pytest.raises(pe.PeError) as err:
+                    gu.gpu_eval(g, assign, order, flags=flags)
+                assert err.value.code == pe.PE_ERR_UNSUPPORTED
+                continue
             gu.check(g, w, assign, order, flags=flags, label=f"u32 {name}")
     finally:
         g.close()
