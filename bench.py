@@ -127,11 +127,31 @@ def time_oracle(w, assign, order, target_s, threads):
     while True:
         a = np.ascontiguousarray(assign[:, :n]); o = np.ascontiguousarray(order[:, :n])
         t0 = time.perf_counter()
-        orc.evaluate(w, a, o, threads=threads)
+        ref = orc.evaluate(w, a, o, threads=threads)
         dt = max(time.perf_counter() - t0, 1e-6)
         if n >= K or dt >= 0.4 * target_s:
-            return n, dt
+            return n, dt, ref
         n = int(min(K, max(2 * n, n * min(16.0, 0.8 * target_s / dt))))
+
+
+def compare_with_oracle(gpu, ref, n):
+    """Element-by-element comparison of the timed run's outputs (first n candidates) with the oracle's:
+    every array of every valid candidate, the two validity bits of the others."""
+    invalid_bits = 3
+    gst = gpu["status"][:n].view(np.uint32)
+    rst = ref["status"]
+    bad = (rst & invalid_bits) != 0
+    mism = int(np.count_nonzero((gst & invalid_bits) != (rst & invalid_bits)))
+    ok = ~bad
+    mism += int(np.count_nonzero(gst[ok] != rst[ok]))
+    arrays = 1
+    for key in ("makespan", "busy", "peak_mem", "start", "finish"):
+        if key not in gpu or ref.get(key) is None:
+            continue
+        a = gpu[key][..., :n]
+        mism += int(np.count_nonzero(a[..., ok] != ref[key][..., ok]))
+        arrays += 1
+    return {"candidates": int(n), "arrays": arrays, "mismatches": mism, "against": "oracle, element by element"}
 
 
 def run_reference(args):
@@ -146,7 +166,7 @@ def run_reference(args):
     per_step = budget_s / (args.steps + args.warmup)
     K_gen = int(min(w.num_candidates, 8192))
     assign, order = wl.make_candidates(w, K=K_gen)
-    n, dt = time_oracle(w, assign, order, min(per_step, 10.0) * 0.8, threads)   # sizes the per-step sample
+    n, dt, _ = time_oracle(w, assign, order, min(per_step, 10.0) * 0.8, threads)   # sizes the per-step sample
     if n > K_gen:
         n = K_gen
     from oracle import pe_oracle as orc
@@ -163,8 +183,9 @@ def run_reference(args):
         "plans_per_s": value / V, "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int32", "data": "synthetic",
-        "config": {"workload": args.workload, "V": V, "D": D, "E": w.num_edges, "K": w.num_candidates,
-                   "outputs": "full", "sample": f"{n} candidates per step"},
+        "config": {"workload": args.workload, "V": V, "E": w.num_edges, "D": D, "L": w.num_link_classes,
+                   "K_per_gpu": w.num_candidates, "outputs": "full", "order_bytes": 2 if V <= 65536 else 4,
+                   "sample": f"the oracle evaluates {n} of the {w.num_candidates} candidates per step"},
         "cpu_baseline": {"value": value, "unit": "op-evals/s", "cores": threads, "kind": "oracle",
                          "sample": f"{n} of {w.num_candidates} candidates per step, {args.steps} steps"},
         "e2e": {"value": value, "unit": "op-evals/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -318,6 +339,10 @@ def run_ours(args):
         raise SystemExit("device-side error word set during the timed region")
     total_ms = max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
+    # outputs of the last timed step, kept for the comparison with the oracle below
+    timed_out = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        timed_out = {k: v.cpu().numpy() for k, v in d_out.items()}
     value = world * K * V / (ms_per_step * 1e-3)
 
     # ---- end to end: host buffers through pe_eval_batch_host, copies inside the timed region ----
@@ -342,6 +367,29 @@ def run_ours(args):
     e2e_value = world * K * V * e2e_steps / max_over_ranks(e2e_s, dev)
     h2d = V * K * (1 + obytes)
     d2h = sum(v.numel() * v.element_size() for v in d_out.values())
+    # the same call when a search loop only wants the summary outputs back (makespan, busy, peak, status)
+    e2e_summary = None
+    if want_times:
+        souts = pe.make_outputs(**{k: v.data_ptr() for k, v in h_out.items() if k not in ("start", "finish")})
+
+        def e2e_summary_step():
+            rc = pe.pe_eval_batch_host(g.handle, K, h_assign.data_ptr(), h_order.data_ptr(), obytes, flags, souts,
+                                       d_assign.data_ptr(), d_order.data_ptr(), outs, ws.data_ptr(), ws_bytes,
+                                       stream.cuda_stream)
+            if rc != pe.PE_OK:
+                raise pe.PeError(rc, "pe_eval_batch_host")
+
+        e2e_summary_step()
+        barrier(); torch.cuda.synchronize(dev)
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e_summary_step()
+        torch.cuda.synchronize(dev)
+        es = time.perf_counter() - t0
+        e2e_summary = {"value": world * K * V * e2e_steps / max_over_ranks(es, dev), "unit": "op-evals/s",
+                       "outputs": "summary", "h2d_bytes_per_step": h2d,
+                       "d2h_bytes_per_step": sum(v.numel() * v.element_size() for k, v in d_out.items()
+                                                 if k not in ("start", "finish")), "steps": e2e_steps}
 
     others = None
     decode = []
@@ -402,12 +450,14 @@ def run_ours(args):
         if rec and rec[0] == kernel_source_hash():
             traffic = rec[1] * K * V
         cpu = None
+        parity = None
         if world == 1 and not args.no_cpu_baseline:
             threads = os.cpu_count() or 1
-            n, dt = time_oracle(w, h_assign.numpy(), h_order.numpy().view(np.uint16 if obytes == 2 else np.uint32),
-                                args.cpu_seconds, threads)
+            n, dt, ref = time_oracle(w, h_assign.numpy(), h_order.numpy().view(np.uint16 if obytes == 2 else np.uint32),
+                                     args.cpu_seconds, threads)
             cpu = {"value": n * V / dt, "unit": "op-evals/s", "cores": threads, "kind": "oracle",
                    "sample": f"first {n} of {K} candidates, all outputs, {dt:.1f} s"}
+            parity = compare_with_oracle(timed_out, ref, n)
         line = {
             "metric": "op_evals_per_s", "value": value, "unit": "op-evals/s", "plans_per_s": value / V,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
@@ -421,7 +471,8 @@ def run_ours(args):
                          "kernel_ms": kms, "algorithmic_bytes_per_launch": alg},
             "e2e": {"value": e2e_value, "unit": "op-evals/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
-            "gpu_launches": launches, "clocks": clocks, "cpu_baseline": cpu,
+            "e2e_summary_outputs": e2e_summary,
+            "gpu_launches": launches, "clocks": clocks, "cpu_baseline": cpu, "parity": parity,
         }
         if others is not None:
             for o in others:
@@ -434,6 +485,8 @@ def run_ours(args):
                 o["frac"] = o["gbs"] / peak
             line["exclusive_channels"] = exclusive
         print(json.dumps(line), flush=True)
+        if parity is not None and parity["mismatches"] != 0:
+            raise SystemExit(f"the timed run's outputs differ from the oracle: {parity}")
     g.close()
     if world > 1:
         dist.destroy_process_group()

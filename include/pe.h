@@ -186,8 +186,10 @@ int pe_eval_batch_host(pe_graph* g, int64_t K, const uint8_t* host_assign, const
 int pe_eval_batch_noalloc(pe_graph* g, int64_t K, const uint8_t* assign, const void* order, int order_bytes,
                           uint32_t flags, const pe_outputs* out, void* cuda_stream);
 
-/* Priority-list decoding: the step in front of pe_eval_batch (Section IV: heuristics for this problem are
- * "priority dispatch rule-based algorithms"; Eq. 8 needs the resulting order to be consistent with B).
+/* Priority-list decoding: the step in front of pe_eval_batch.  The paper prints no decoder from a priority
+ * list to (x, pi); Section IV mentions dispatch rules only as the inspiration of its coarsening heuristic.
+ * The rule below is this library's choice; what the model requires is that the resulting order be
+ * consistent with B (Eq. 8).
  * A candidate ranks the operators through a list; the priority order is then built position by position:
  * among the operators not yet placed whose predecessors in B have all been placed, the one of smallest rank
  * comes next.  The result is a topological order of G_m - a valid `order` argument of pe_eval_batch - and a

@@ -197,8 +197,9 @@ extern "C" int pe_oracle_eval(int32_t V, int32_t E, const int32_t* edge_src, con
 // ---------------------------------------------------------------------------------------------
 // Priority-list decoding: the step before evaluation.  TEST INFRASTRUCTURE ONLY, like the rest.
 //
-// Section IV frames heuristics for this problem as "priority dispatch rule-based algorithms".
-// The rule written out here: a candidate gives every operation a priority rank through a list
+// The paper prints no decoder from a priority list to an order; Section IV mentions dispatch rules
+// only as the inspiration of its coarsening heuristic.  The rule written out here (a choice of
+// this repository, consistent with Eq. 8): a candidate gives every operation a priority rank through a list
 // (list[r] = the operation of rank r, rank 0 the most urgent; any permutation of I, it need not
 // respect the precedence edges B), and the priority order pi is built one position at a time:
 // among the operations not yet placed whose predecessors in B have all been placed, the one of

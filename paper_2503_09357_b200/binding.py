@@ -283,6 +283,8 @@ class Graph:
                                 ws.data_ptr(), n, s)
         if rc != PE_OK:
             raise PeError(rc, "pe_decode_priority")
+        if stream is not None:        # the workspace dies here: keep the allocator from reusing it under the kernel
+            ws.record_stream(torch.cuda.ExternalStream(stream, device=dev))
         return order, status
 
     def eval_batch(self, assign, order, flags=0, out=None, workspace=None, want_times=True, stream=None):
@@ -303,4 +305,6 @@ class Graph:
                            ws.data_ptr(), ws_bytes, s)
         if rc != PE_OK:
             raise PeError(rc, "pe_eval_batch")
+        if stream is not None:        # a workspace allocated here dies here: keep the allocator from reusing it
+            ws.record_stream(torch.cuda.ExternalStream(stream, device=torch.device("cuda", self.device)))
         return out

@@ -1,7 +1,7 @@
 // pe_decode_priority: priority-list decoding, the step in front of pe_eval_batch.
 //
-// Section IV of the paper frames heuristics for the planning problem as priority dispatch
-// rules.  The rule implemented here: a candidate ranks the operators through a list (list[r] =
+// The paper prints no decoder (Section IV mentions dispatch rules only as the inspiration of its
+// coarsening heuristic); the rule implemented here is this library's choice: a candidate ranks the operators through a list (list[r] =
 // the operator of rank r; any permutation of I), and the priority order pi is built position by
 // position: among the operators not yet placed whose predecessors in B have all been placed, the
 // one of smallest rank comes next (Kahn's algorithm with the ranks as priorities).  The result is

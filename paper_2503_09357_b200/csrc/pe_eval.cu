@@ -7,7 +7,9 @@
 // machine's memory level moves by A_i (Eqs. 16-19).  The variants differ in where the
 // per-candidate state lives and how lanes map to candidates.
 #include <atomic>
+#include <map>
 #include <mutex>
+#include <utility>
 #include <climits>
 #include <cstdio>
 
@@ -20,6 +22,19 @@
 namespace pe {
 
 static std::atomic<int64_t> g_launches{0};
+
+bool raise_smem_limit(const void* func, size_t bytes) {
+  static std::mutex mu;
+  static std::map<std::pair<int, const void*>, size_t> limit;   // (device, kernel) -> bytes granted so far
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  std::lock_guard<std::mutex> lock(mu);
+  size_t& cur = limit[std::make_pair(dev, func)];
+  if (bytes <= cur) return true;
+  if (cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return false;
+  cur = bytes;
+  return true;
+}
 
 // ============================================================================================
 // Variant GLOBAL: one thread per candidate; end time of every operator in the caller's
@@ -311,11 +326,12 @@ static bool plan_warp(const pe_graph* g, int64_t K, uint32_t flags, bool allow_c
 // in the workspace, a chunk of candidates at a time; a chunk is sixteen times what the GPU holds at once.
 static bool plan_team(const pe_graph* g, int64_t K, bool allow_compact, Plan* p) {
   if (!g->narrow_ok || !allow_compact || g->max_indeg > 3 || g->time_bound >= (int64_t)1 << 23) return false;
-  const size_t smem = round_up((size_t)4 * (g->V + 1) + (size_t)4 * (5 * g->D + 2), 16);
+  size_t smem = round_up((size_t)4 * (g->V + 2) + (size_t)4 * (5 * g->D + 2), 16);
+  if (const char* e = std::getenv("PE_TEAM_PAD")) smem += (size_t)std::atoi(e);
   if (smem > g->smem_optin) return false;
   int nw = 6;
   if (const char* e = std::getenv("PE_TEAM_WARPS")) nw = std::atoi(e);
-  if (nw != 2 && nw != 4 && nw != 6) return false;
+  if (nw != 4 && nw != 6) return false;
   p->variant = PE_VARIANT_TEAM;
   p->threads = 32 * nw;
   p->smem = smem;
@@ -410,9 +426,14 @@ static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, bool allow_co
       // for the largest graphs the global-state kernel, which is bound by random DRAM accesses but
       // keeps thousands of candidates in flight, is faster.
       if (plan_shared(g, allow_compact, p) && p->threads >= 48) return PE_OK;
-      Plan w, gl;
+      Plan w, gl, tm;
       const bool has_w = plan_warp(g, K, flags, allow_compact, &w);
       const bool has_g = plan_global(g, K, flags, allow_compact, &gl);
+      // Once fewer than about twenty single-warp candidates fit on an SM, a block of warps per candidate
+      // is faster (measured at V = 4096: 3.6e10 against 2.6e10 operator-evaluations/s at D = 64, 2.7e10
+      // against 2.0e10 at D = 8; at V = 16384: 3.1e10 against 1.0e10 (warp) and 2.3e10 against 1.25e10
+      // (global); at V = 1024 the single-warp kernel still wins, 4.0e10 against 3.0e10).
+      if (plan_team(g, K, allow_compact, &tm) && (!has_w || w.threads < 20 * 32)) { *p = tm; return PE_OK; }
       // With three warps per SM the two are close; the global-state kernel loses once it has to keep the
       // per-machine records in the workspace as well (measured at V = 16384: 1.25e10 against 0.84e10
       // operator-evaluations/s at D = 8, 0.93e10 against 1.01e10 at D = 64).

@@ -73,8 +73,8 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
   const int64_t c = blockIdx.x;
   const uint32_t vmax = (uint32_t)(V - 1), dmax = (uint32_t)(D - 1);
 
-  uint32_t* state = reinterpret_cast<uint32_t*>(smem_raw);   // [V + 1]
-  int32_t* free_at = reinterpret_cast<int32_t*>(state + V + 1);
+  uint32_t* state = reinterpret_cast<uint32_t*>(smem_raw);   // [V + 2]: row V the sentinel (always 0), row V + 1 a dump
+  int32_t* free_at = reinterpret_cast<int32_t*>(state + V + 2);   // = state[V + 2 + machine]
   int32_t* lvl = free_at + D;
   int32_t* peak = lvl + D;
   int32_t* busy = peak + D;
@@ -190,13 +190,15 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
   int32_t* start_col = TIMES ? out.start + (size_t)c * sd.out_cand : nullptr;
   int32_t* finish_col = TIMES ? out.finish + (size_t)c * sd.out_cand : nullptr;
 
+  // order entries two of this warp's windows ahead, operator records one ahead
   auto load_order = [&](int win) -> uint32_t {
     const int k = win * 32 + lane;
-    return k < V ? (uint32_t)order_col[(size_t)k * sd.in_row] : 0u;
+    if (k >= V) return 0u;
+    return STAGED ? (uint32_t)order_col[k] : (uint32_t)order_col[(size_t)k * sd.in_row];
   };
-  // order entries two of this warp's windows ahead, operator records one ahead
   uint32_t o_cur = load_order(warp), o_nxt = load_order(warp + NW);
   uint4 rec_nxt = __ldg(gp.ops + min(o_cur, vmax));
+  const uint32_t none = (uint32_t)V;
 
   for (int win = warp; win < nwin; win += NW) {
     const int base = win * 32;
@@ -209,13 +211,15 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
     rec_nxt = __ldg(gp.ops + min(o_cur, vmax));
 
     // ---- set-up: nothing here depends on a time ----
-    if (act) order_max = max(order_max, iu);
-    const uint32_t i = act ? min(iu, vmax) : (uint32_t)V;
+    const uint32_t i = act ? min(iu, vmax) : none;
     const uint32_t own = state[i];
-    if (act && (own >> 8) != ((kTeamPending >> 8) | (uint32_t)k)) st |= PE_STATUS_ORDER_INVALID;  // repeated operator
     const uint32_t jr = own & 0xFFu;
-    if (!BY_POS && act) dev_max = max(dev_max, jr);
     const uint32_t j = min(jr, dmax);
+    if (act) {
+      order_max = max(order_max, iu);
+      if (!BY_POS) dev_max = max(dev_max, jr);
+      if ((own >> 8) != ((kTeamPending >> 8) | (uint32_t)k)) st |= PE_STATUS_ORDER_INVALID;   // repeated operator
+    }
     const int indeg = (int)(rec.y >> 24);
     const int32_t dur = act ? (int32_t)(rec.y & 0xFFFFu) : 0;
     const int32_t dA = act ? (int32_t)(rec.y << 8) >> 24 : 0;
@@ -223,19 +227,22 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
     // previous / last operator of the same machine inside the window (Eqs. 7-8)
     const uint32_t same_dev = __match_any_sync(FULL, act ? j : (0x100u | lane));
     const uint32_t below = same_dev & lt_mask;
-    const int prev = below ? 31 - __clz(below) : -1;
+    const bool has_prev = below != 0;
     const bool last_on_dev = (same_dev >> lane) == 1u;
 
-    // incoming edges: edge q owns slot q.  A source inside the window becomes (lane, delay) for the
+    // Incoming edges: edge q owns slot q.  A source inside the window becomes (lane, delay) for the
     // relaxation; any other becomes (state address, delay) for the gather under the baton.  The unused
     // half of a slot is neutral: lane = own lane with delay kNever, address = sentinel with delay kNever.
-    const uint32_t none = (uint32_t)V;
-    uint32_t a0 = none, a1 = none, a2 = none;
-    int32_t g0 = kNever, g1 = kNever, g2 = kNever;
-    int l0 = lane, l1 = lane, l2 = lane;
-    int32_t d0 = kNever, d1 = kNever, d2 = kNever;
+    // `rel` is the source's position relative to the window when its word is pending; a final word
+    // (bit 31 clear) wraps to a huge value, so one unsigned compare tells "inside the window, before me".
+    const uint32_t pend_base = (kTeamPending >> 8) + (uint32_t)base;
     uint32_t depmask = 0;
-    auto delay_of = [&](uint32_t lo, uint32_t hi, uint32_t w) -> uint32_t {
+    uint32_t a0, a1, a2;
+    int32_t g0, g1, g2, d0, d1, d2;
+    int l0, l1, l2;
+    auto classify = [&](uint32_t lo, uint32_t hi, uint32_t& addr, int32_t& gdel, int& lsl, int32_t& ldel) {
+      const uint32_t p = lo & 0xFFFFu;
+      const uint32_t w = state[p];
       const uint32_t xp = w & 0xFFu;
       uint32_t delay = lo >> 16;
       if (NEED_CLS) {
@@ -243,58 +250,48 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
         if (TWO_CLASS) delay = cl == 1u ? hi : delay;
         if (cl == 0xFFu) {
           delay = 0;
-          if ((lo & 0xFFFFu) != none && xp != j) st |= PE_STATUS_NO_CHANNEL;
+          if (p != none && xp != j) st |= PE_STATUS_NO_CHANNEL;
         }
       }
-      return xp != j ? delay : 0u;
+      const int32_t dly = xp != j ? (int32_t)delay : 0;
+      const uint32_t rel = (w >> 8) - pend_base;
+      const bool inw = rel < (uint32_t)lane;
+      if (!inw && rel < 0x10000u) st |= PE_STATUS_ORDER_INVALID;   // pending, but not before this operator
+      addr = inw ? none : p;
+      gdel = inw ? kNever : dly;
+      lsl = inw ? (int)rel : lane;
+      ldel = (inw ? dly : kNever) + dur;   // D^o folded into the in-window delays (Eq. 3)
+      depmask |= inw ? 1u << rel : 0u;
     };
-    auto classify = [&](uint32_t lo, uint32_t hi, uint32_t& addr, int32_t& gdel, int& lsl, int32_t& ldel) {
-      const uint32_t p = lo & 0xFFFFu;
-      const uint32_t w = state[p];
-      const int32_t dly = (int32_t)delay_of(lo, hi, w);
-      const uint32_t pos = (w >> 8) & 0xFFFFu;
-      if ((w & kTeamPending) && pos >= (uint32_t)base) {
-        if (pos < (uint32_t)k) {
-          lsl = (int)(pos - (uint32_t)base);
-          ldel = dly;
-          depmask |= 1u << lsl;
-        } else {
-          st |= PE_STATUS_ORDER_INVALID;   // a predecessor that is not before this operator
-        }
-      } else {
-        addr = p;   // final already, or in an earlier window: final by the time the baton arrives
-        gdel = dly;
-      }
-    };
-    if (act) {
-      classify(rec.z, rec.w, a0, g0, l0, d0);
-      if (TWO_CLASS) {
-        const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
-        if (indeg > 1) { const uint2 e1 = __ldg(ed + 1); classify(e1.x, e1.y, a1, g1, l1, d1); }
-        if (indeg > 2) { const uint2 e2 = __ldg(ed + 2); classify(e2.x, e2.y, a2, g2, l2, d2); }
-      } else {
-        classify(rec.w, 0u, a1, g1, l1, d1);
-        classify(rec.x, 0u, a2, g2, l2, d2);
-      }
+    // (a lane beyond the end of the order goes through the same code on operator 0's record; what it
+    //  classifies and flags is dropped right after)
+    const uint32_t st_before = st;
+    classify(rec.z, rec.w, a0, g0, l0, d0);
+    if (TWO_CLASS) {
+      a1 = none; a2 = none; g1 = kNever; g2 = kNever; l1 = lane; l2 = lane; d1 = kNever + dur; d2 = kNever + dur;
+      const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
+      if (indeg > 1) { const uint2 e1 = __ldg(ed + 1); classify(e1.x, e1.y, a1, g1, l1, d1); }
+      if (indeg > 2) { const uint2 e2 = __ldg(ed + 2); classify(e2.x, e2.y, a2, g2, l2, d2); }
+    } else {
+      classify(rec.w, 0u, a1, g1, l1, d1);
+      classify(rec.x, 0u, a2, g2, l2, d2);
     }
-    int lp = lane;
-    int32_t dp = kNever;
-    if (act && prev >= 0) { lp = prev; dp = 0; depmask |= 1u << prev; }
-    // Depth of the window: peel off, round by round, the lanes whose sources are all peeled.  After r
-    // rounds of relaxation every lane of depth <= r holds its final value, so the number of rounds the
-    // baton has to wait for is known before it arrives and the loop under it needs no vote.
+    if (!act) { st = st_before; depmask = 0; a0 = a1 = a2 = none; }
+    const int prev = 31 - __clz(below);
+    const int lp = has_prev ? prev : lane;
+    const int32_t dp = (has_prev ? 0 : kNever) + dur;
+    depmask |= has_prev ? 1u << prev : 0u;
+    // Depth of the window: peel off, round by round, the lanes whose sources are all peeled.  After n
+    // rounds of relaxation every lane of depth <= n holds its final value, so the number of rounds is
+    // known before the baton arrives and the loop under it needs no vote.
     int nrounds = 0;
     {
-      bool fin = depmask == 0;
-      uint32_t done = __ballot_sync(FULL, fin);
+      uint32_t done = __ballot_sync(FULL, depmask == 0);
       while (done != FULL) {
-        fin = fin || (depmask & ~done) == 0;
-        done = __ballot_sync(FULL, fin);
+        done = __ballot_sync(FULL, (depmask & ~done) == 0);
         ++nrounds;
       }
     }
-    // e_l = max(r_base, max_q(e_src(q) + delay_q)) + D^o (Eqs. 3, 7-8, 11-13) with D^o folded into the delays
-    d0 += dur; d1 += dur; d2 += dur; dp += dur;
 
     // ---- memory levels (Eqs. 17-19): prefix sums of A along each machine's lanes, then the machine's
     // level before the window, under the ledger baton ----
@@ -302,9 +299,10 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
     {
       uint32_t m = below;
       while (__any_sync(FULL, m != 0)) {
-        const int src = m ? __ffs(m) - 1 : lane;
-        const int32_t a_src = __shfl_sync(FULL, dA, src);
-        if (m) { lv += a_src; m &= m - 1; }
+        const int top = 31 - __clz(m);   // (-1 when m == 0: the shuffle then reads lane 31 and the value is dropped)
+        const int32_t a_src = __shfl_sync(FULL, dA, top);
+        lv += m ? a_src : 0;
+        m &= ~(1u << (top & 31));
       }
     }
     if (act) {
@@ -322,34 +320,35 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
     if (win + 1 < nwin) named_arrive(1 + NW + next_warp, 64);
 
     // ---- times, under the baton: every earlier window is final ----
+    // (all accesses under the baton are unconditional: a lane with nothing to read reads the sentinel,
+    //  a lane with nothing to write writes the dump row, so the warp never diverges here)
+    const uint32_t fr_at = (act && !has_prev) ? (uint32_t)(V + 2) + j : none;            // machine free since
+    const uint32_t st_at = act ? i : none + 1u;                                           // own state word
+    const uint32_t fw_at = (act && last_on_dev) ? (uint32_t)(V + 2) + j : none + 1u;      // machine free from
     if (win > 0) named_sync(1 + warp, 64);
     const uint32_t w0 = state[a0], w1 = state[a1], w2 = state[a2];
-    int32_t r_base = (act && prev < 0) ? free_at[j] : 0;
-    r_base = max(r_base, (int32_t)(w0 >> 8) + g0);
-    r_base = max(r_base, (int32_t)(w1 >> 8) + g1);
-    r_base = max(r_base, (int32_t)(w2 >> 8) + g2);
+    const int32_t fr = (int32_t)state[fr_at];
+    const int32_t r_base = __vimax3_s32(__viaddmax_s32((int32_t)(w0 >> 8), g0, fr), (int32_t)(w1 >> 8) + g1,
+                                        (int32_t)(w2 >> 8) + g2);
     const int32_t b_end = r_base + dur;
     int32_t e = b_end;
     // every dependence points to a lower lane, so the values rise monotonically to the window's
     // longest-path solution, which they reach after `nrounds` rounds
     for (int it = 0; it < nrounds; ++it) {
-      const int32_t t0 = __shfl_sync(FULL, e, l0) + d0;
-      const int32_t t1 = __shfl_sync(FULL, e, l1) + d1;
-      const int32_t t2 = __shfl_sync(FULL, e, l2) + d2;
-      const int32_t t3 = __shfl_sync(FULL, e, lp) + dp;
-      e = max(max(b_end, t0), max(max(t1, t2), t3));
+      const int32_t s0 = __shfl_sync(FULL, e, l0), s1 = __shfl_sync(FULL, e, l1);
+      const int32_t s2 = __shfl_sync(FULL, e, l2), s3 = __shfl_sync(FULL, e, lp);
+      e = __vimax3_s32(__viaddmax_s32(s0, d0, b_end), __viaddmax_s32(s1, d1, s2 + d2), s3 + dp);
     }
-    if (act) {
-      state[i] = ((uint32_t)e << 8) | j;
-      if (last_on_dev) free_at[j] = e;
-    }
+    state[st_at] = ((uint32_t)e << 8) | j;
+    state[fw_at] = (uint32_t)e;
     __syncwarp();
     if (win + 1 < nwin) named_arrive(1 + next_warp, 64);
 
     // ---- after the baton has gone: outputs ----
     z = max(z, e);
     if (TIMES && act) {
-      const size_t at = (size_t)(by_op_times ? i : (uint32_t)k) * sd.out_row;
+      const uint32_t row = by_op_times ? i : (uint32_t)k;
+      const size_t at = STAGED ? (size_t)row : (size_t)row * sd.out_row;
       start_col[at] = e - dur;
       finish_col[at] = e;
     }

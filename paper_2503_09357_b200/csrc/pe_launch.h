@@ -28,9 +28,15 @@ struct Plan {
   size_t team_off_order = 0, team_off_assign = 0, team_off_start = 0, team_off_finish = 0;   // offsets in the workspace
 };
 
+// Raise a kernel's dynamic shared-memory limit to at least `bytes` on the current device.  The attribute
+// belongs to the function, not to a launch, and several host threads may launch the same kernel with
+// different sizes: the limit is therefore only ever raised, under a lock, so a launch that was prepared
+// with a smaller size can never find the limit lowered underneath it.
+bool raise_smem_limit(const void* func, size_t bytes);
+
 template <typename Kern>
 static bool set_smem(Kern kern, size_t bytes) {
-  return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
+  return raise_smem_limit(reinterpret_cast<const void*>(kern), bytes);
 }
 
 // pe_eval_lane_kernel: state in shared memory (plan variant SHARED) or in `gstate` (GLOBAL).

@@ -65,6 +65,16 @@ extern "C" int pe_select_best(int64_t K, const int32_t* makespan, const uint32_t
                               int64_t* result, void* cuda_stream) {
   if (K < 0 || !result || (K > 0 && (!makespan || !status))) return PE_ERR_INVALID_ARG;
   if (K > 0xFFFFFFFFll) return PE_ERR_INVALID_ARG;  // the index shares a 64-bit key with the makespan
+  // run on the device that owns `result` (the other arrays must live there too)
+  cudaPointerAttributes attr;
+  if (cudaPointerGetAttributes(&attr, result) != cudaSuccess ||
+      (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged)) {
+    cudaGetLastError();
+    return PE_ERR_INVALID_ARG;
+  }
+  int prev = -1;
+  if (cudaGetDevice(&prev) != cudaSuccess) return PE_ERR_CUDA;
+  if (prev != attr.device && cudaSetDevice(attr.device) != cudaSuccess) return PE_ERR_CUDA;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   unsigned long long* scratch = reinterpret_cast<unsigned long long*>(result);
   pe::pe_select_init_kernel<<<1, 1, 0, stream>>>(scratch);
@@ -72,5 +82,7 @@ extern "C" int pe_select_best(int64_t K, const int32_t* makespan, const uint32_t
   if (blocks > 1184) blocks = 1184;  // 148 SMs x 8 resident blocks: a grid-stride loop covers the rest
   if (blocks < 1) blocks = 1;
   pe::pe_select_kernel<<<blocks, 256, 0, stream>>>(K, makespan, status, reject_mask, scratch);
-  return cudaGetLastError() == cudaSuccess ? PE_OK : PE_ERR_CUDA;
+  const int ret = cudaGetLastError() == cudaSuccess ? PE_OK : PE_ERR_CUDA;
+  if (prev != attr.device) cudaSetDevice(prev);
+  return ret;
 }

@@ -46,7 +46,6 @@ int launch2(const TeamCall& t) {
 template <bool BY_POS>
 int launch1(const TeamCall& t) {
   switch (t.p->threads / 32) {
-    case 2: return launch2<2, BY_POS>(t);
     case 4: return launch2<4, BY_POS>(t);
     case 6: return launch2<6, BY_POS>(t);
     default: return PE_ERR_UNSUPPORTED;
