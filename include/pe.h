@@ -221,6 +221,43 @@ int pe_decode_priority(pe_graph* g, int64_t K, const void* list, int order_bytes
 int pe_select_best(int64_t K, const int32_t* makespan, const uint32_t* status, uint32_t reject_mask, int64_t* result,
                    void* cuda_stream);
 
+/* Operator merging in front of candidate generation (Section IV, Algorithm 1): shrinks G_m(I, B) to at most
+ * `target_ops` operators by repeatedly merging pairs, so that a search (or the paper's MIP) works on a graph
+ * of manageable size.  Host-only: every pointer is a HOST pointer and no GPU is touched.
+ *
+ * The algorithm alternates two loops until |I| <= target_ops or a whole pass merges nothing: merges of pairs
+ * joined by an edge, then merges of pairs not joined by a path.  Before candidates are looked for, the
+ * topologically redundant edges {(i1, i2) in B : some i3 has (i1, i3) and (i3, i2) in B} are set aside
+ * (Section IV's definition); merging works on the full edge set.
+ *   - edge candidate: an edge (u, v) of the remaining graph where v has a single input and u a single output,
+ *     merged duration <= max_dur_edge and merged memory requirement <= max_mem_edge.  Safe: no cycle can
+ *     arise and the critical path keeps its length (Section IV).
+ *   - non-edge candidate: two operators with no directed path between them in either direction (the paper says
+ *     "without a direct edge"; incomparability is what rules out a cycle), within max_dur_nonedge and
+ *     max_mem_nonedge - the stricter thresholds Section IV asks for are the caller's to choose.
+ *   - among several candidates the one with the smallest merged duration goes first, ties to the smallest
+ *     (u, v), a group being identified by its smallest operator (the paper does not say).
+ *   - a merged operator's duration, A and W are the sums over its members (Section IV); it inherits every edge
+ *     to or from a third operator; edges that become parallel (also duplicate input edges) are combined into
+ *     one whose communication duration per link class is the larger of the two.  The memory requirement
+ *     tested against the thresholds is W + max(A, 0) summed over the members (the paper gives no formula).
+ * Outputs (caller-allocated): op_map [V] = merged operator of every original one, merged operators numbered in
+ * the order of their smallest member; *num_ops_out, *num_edges_out; edge_src / edge_dst [E], comm [E * L]
+ * (NULL allowed if the input has no comm), sorted by (source, destination); dur [V]; mem_delta, mem_weight [V]
+ * (each may be NULL).  Only the first *num_ops_out / *num_edges_out entries are written.  The result is a
+ * DAG and can go straight into pe_graph_create.  V above 16384 is PE_ERR_UNSUPPORTED (the adjacency is kept
+ * as two V x V bit matrices); the description is validated first (PE_ERR_CYCLE, PE_ERR_RANGE, ...). */
+typedef struct {
+  int32_t target_ops;      /* N >= 1: stop once |I| <= N */
+  int32_t max_dur_edge;    /* thresholds of merges along an edge */
+  int32_t max_mem_edge;
+  int32_t max_dur_nonedge; /* thresholds of merges of unrelated operators */
+  int32_t max_mem_nonedge;
+} pe_coarsen_params;
+int pe_coarsen(const pe_graph_desc* desc, const pe_coarsen_params* prm, int32_t* op_map, int32_t* num_ops_out,
+               int32_t* num_edges_out, int32_t* edge_src, int32_t* edge_dst, int32_t* comm, int32_t* dur,
+               int32_t* mem_delta, int32_t* mem_weight);
+
 /* Synchronise `cuda_stream` and return the graph's device-side error word: PE_OK, or
  * PE_ERR_TIMEOUT if a kernel gave up a bounded wait (its outputs are then invalid).  Clears the word. */
 int pe_graph_poll_error(pe_graph* g, void* cuda_stream);

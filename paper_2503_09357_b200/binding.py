@@ -82,6 +82,15 @@ _lib.pe_strerror.restype = ctypes.c_char_p
 _lib.pe_strerror.argtypes = [ctypes.c_int]
 
 
+class pe_coarsen_params(ctypes.Structure):
+    _fields_ = [("target_ops", ctypes.c_int32), ("max_dur_edge", ctypes.c_int32), ("max_mem_edge", ctypes.c_int32),
+                ("max_dur_nonedge", ctypes.c_int32), ("max_mem_nonedge", ctypes.c_int32)]
+
+
+_lib.pe_coarsen.restype = ctypes.c_int
+_lib.pe_coarsen.argtypes = [ctypes.POINTER(pe_graph_desc), ctypes.POINTER(pe_coarsen_params)] + [_P] * 9
+
+
 class PeError(RuntimeError):
     def __init__(self, code, where):
         self.code = code
@@ -123,6 +132,27 @@ def desc_from_workload(w):
     return make_desc(w.num_ops, w.edge_src, w.edge_dst, w.dur, w.num_devices, mem_delta=w.mem_delta,
                      mem_weight=w.mem_weight, num_link_classes=w.num_link_classes, link_class=w.link_class,
                      comm=w.comm, mem_capacity=w.mem_capacity)
+
+
+def pe_coarsen(desc, target_ops, max_dur_edge, max_mem_edge, max_dur_nonedge, max_mem_nonedge):
+    """Algorithm 1 on a host description (argument marshalling only).  Returns a dict of numpy arrays
+    (op_map, edge_src, edge_dst, comm [E', L], dur, mem_delta, mem_weight) and num_ops."""
+    V, E, L = int(desc.num_ops), int(desc.num_edges), int(desc.num_link_classes)
+    prm = pe_coarsen_params(int(target_ops), int(max_dur_edge), int(max_mem_edge), int(max_dur_nonedge),
+                            int(max_mem_nonedge))
+    op_map = np.zeros(max(V, 1), np.int32)
+    n_ops, n_edges = ctypes.c_int32(0), ctypes.c_int32(0)
+    src, dst = np.zeros(max(E, 1), np.int32), np.zeros(max(E, 1), np.int32)
+    comm = np.zeros(max(E * L, 1), np.int32)
+    dur, A, W = (np.zeros(max(V, 1), np.int32) for _ in range(3))
+    rc = _lib.pe_coarsen(ctypes.byref(desc), ctypes.byref(prm), op_map.ctypes.data, ctypes.addressof(n_ops),
+                         ctypes.addressof(n_edges), src.ctypes.data, dst.ctypes.data, comm.ctypes.data,
+                         dur.ctypes.data, A.ctypes.data, W.ctypes.data)
+    if rc != PE_OK:
+        raise PeError(rc, "pe_coarsen")
+    n, m = n_ops.value, n_edges.value
+    return dict(num_ops=n, op_map=op_map[:V], edge_src=src[:m], edge_dst=dst[:m], comm=comm[:m * L].reshape(m, L),
+                dur=dur[:n], mem_delta=A[:n], mem_weight=W[:n])
 
 
 def pe_graph_validate(desc) -> int:

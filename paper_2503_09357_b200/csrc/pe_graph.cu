@@ -236,7 +236,12 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
       ok = cudaStreamCreateWithFlags(&g->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
            cudaStreamCreateWithFlags(&g->copy_out, cudaStreamNonBlocking) == cudaSuccess &&
            cudaEventCreateWithFlags(&g->ev_begin, cudaEventDisableTiming) == cudaSuccess &&
-           cudaEventCreateWithFlags(&g->ev_end, cudaEventDisableTiming) == cudaSuccess;
+           cudaEventCreateWithFlags(&g->ev_end, cudaEventDisableTiming) == cudaSuccess &&
+           cudaStreamCreateWithFlags(&g->team_stream[0], cudaStreamNonBlocking) == cudaSuccess &&
+           cudaStreamCreateWithFlags(&g->team_stream[1], cudaStreamNonBlocking) == cudaSuccess &&
+           cudaEventCreateWithFlags(&g->team_fork, cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&g->team_join[0], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&g->team_join[1], cudaEventDisableTiming) == cudaSuccess;
       for (int q = 0; ok && q < pe_graph::kMaxChunks; ++q)
         ok = cudaEventCreateWithFlags(&g->ev_in[q], cudaEventDisableTiming) == cudaSuccess &&
              cudaEventCreateWithFlags(&g->ev_done[q], cudaEventDisableTiming) == cudaSuccess;
@@ -253,6 +258,11 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
     if (g->copy_out) cudaStreamDestroy(g->copy_out);
     if (g->ev_begin) cudaEventDestroy(g->ev_begin);
     if (g->ev_end) cudaEventDestroy(g->ev_end);
+    for (int q = 0; q < 2; ++q) {
+      if (g->team_stream[q]) cudaStreamDestroy(g->team_stream[q]);
+      if (g->team_join[q]) cudaEventDestroy(g->team_join[q]);
+    }
+    if (g->team_fork) cudaEventDestroy(g->team_fork);
     for (int q = 0; q < pe_graph::kMaxChunks; ++q) {
       if (g->ev_in[q]) cudaEventDestroy(g->ev_in[q]);
       if (g->ev_done[q]) cudaEventDestroy(g->ev_done[q]);
@@ -274,6 +284,8 @@ extern "C" int pe_destroy(pe_graph* g) {
   cudaStreamDestroy(g->copy_out);
   cudaEventDestroy(g->ev_begin);
   cudaEventDestroy(g->ev_end);
+  for (int q = 0; q < 2; ++q) { cudaStreamDestroy(g->team_stream[q]); cudaEventDestroy(g->team_join[q]); }
+  cudaEventDestroy(g->team_fork);
   for (int q = 0; q < pe_graph::kMaxChunks; ++q) { cudaEventDestroy(g->ev_in[q]); cudaEventDestroy(g->ev_done[q]); }
   bool ok = cudaFree(g->d_blob) == cudaSuccess && cudaFree(g->d_error) == cudaSuccess;
   if (g->d_nblob) ok = cudaFree(g->d_nblob) == cudaSuccess && ok;

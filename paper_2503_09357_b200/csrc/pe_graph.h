@@ -94,6 +94,12 @@ struct pe_graph {
   cudaStream_t copy_in, copy_out;
   cudaEvent_t ev_begin, ev_end, ev_in[kMaxChunks], ev_done[kMaxChunks];
   std::mutex host_mutex;
+  // pe_eval_batch with the TEAM variant works through chunks of candidates; consecutive chunks alternate
+  // between two side streams so that the staging transpositions of one overlap the evaluation of the
+  // other.  `team_mutex` serialises the enqueueing of such calls on one graph (they share the events).
+  cudaStream_t team_stream[2];
+  cudaEvent_t team_fork, team_join[2];
+  std::mutex team_mutex;
   int sm_count;
   size_t smem_optin;   // max dynamic shared memory per block
   size_t smem_per_sm;  // shared memory of an SM

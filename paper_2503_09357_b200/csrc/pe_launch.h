@@ -25,7 +25,8 @@ struct Plan {
   bool staged = false;
   int64_t team_chunk = 0;   // candidates per chunk (multiple of 4)
   int64_t team_vp = 0;      // row length of the staging copies: V rounded up to a multiple of 64
-  size_t team_off_order = 0, team_off_assign = 0, team_off_start = 0, team_off_finish = 0;   // offsets in the workspace
+  size_t team_off_order = 0, team_off_assign = 0, team_off_start = 0, team_off_finish = 0;   // offsets in a half
+  size_t team_half = 0;     // bytes of one half of the workspace (two chunks are in flight)
 };
 
 // Raise a kernel's dynamic shared-memory limit to at least `bytes` on the current device.  The attribute
