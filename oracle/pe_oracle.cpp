@@ -67,13 +67,17 @@ constexpr uint32_t kStatusNoChannel = 8u;
 
 }  // namespace
 
-extern "C" int pe_oracle_eval(int32_t V, int32_t E, const int32_t* edge_src, const int32_t* edge_dst,
-                              const int32_t* dur, const int32_t* mem_delta, const int32_t* mem_weight, int32_t D,
-                              int32_t L, const uint8_t* link_class, const int32_t* comm,
-                              const int32_t* mem_capacity, int64_t K, int64_t c_begin, int64_t c_end,
-                              const uint8_t* assign, const void* order, int order_bytes, uint32_t flags,
-                              int32_t* start, int32_t* finish, int32_t* makespan, int32_t* busy, int32_t* peak_mem,
-                              uint32_t* status) {
+// Heterogeneous machines (footnote of Section III: the model extends "by including the machine
+// dimension relating to the operation allocation decisions"): when `dur_by_machine` is given, operation i
+// lasts dur_by_machine[i * D + j] on machine j, i.e. D^o_i of Eq. 3 becomes D^o_{i, x_i}; everything else
+// is unchanged.  With a NULL table this is the homogeneous evaluation.
+extern "C" int pe_oracle_eval_hetero(int32_t V, int32_t E, const int32_t* edge_src, const int32_t* edge_dst,
+                                     const int32_t* dur, const int32_t* dur_by_machine, const int32_t* mem_delta,
+                                     const int32_t* mem_weight, int32_t D, int32_t L, const uint8_t* link_class,
+                                     const int32_t* comm, const int32_t* mem_capacity, int64_t K, int64_t c_begin,
+                                     int64_t c_end, const uint8_t* assign, const void* order, int order_bytes,
+                                     uint32_t flags, int32_t* start, int32_t* finish, int32_t* makespan,
+                                     int32_t* busy, int32_t* peak_mem, uint32_t* status) {
   if (V <= 0 || E < 0 || D <= 0 || D > 255 || L <= 0 || K < 0 || c_begin < 0 || c_end > K) return -1;
   if (order_bytes != 2 && order_bytes != 4) return -1;
   for (int32_t b = 0; b < E; ++b)
@@ -158,11 +162,12 @@ extern "C" int pe_oracle_eval(int32_t V, int32_t E, const int32_t* edge_src, con
         }
         if (t > r) r = t;
       }
+      const int32_t d_i = dur_by_machine ? dur_by_machine[(size_t)i * D + j] : dur[i];  // D^o of i on its machine
       s[i] = r > free_at[j] ? r : free_at[j];  // Eq. 7 with y from pi: after everything earlier on machine j
-      e[i] = s[i] + dur[i];                    // Eq. 3
+      e[i] = s[i] + d_i;                       // Eq. 3
       free_at[j] = e[i];
       done[i] = 1;
-      busy_j[j] += dur[i];
+      busy_j[j] += d_i;
       lvl[j] += mem_delta[i];                  // Eq. 19, handed on along the machine by Eqs. 17-18
       if (lvl[j] > peak[j]) peak[j] = lvl[j];
       if (e[i] > z) z = e[i];                  // Eq. 2
@@ -192,6 +197,18 @@ extern "C" int pe_oracle_eval(int32_t V, int32_t E, const int32_t* edge_src, con
     if (status) status[c] = st;
   }
   return 0;
+}
+
+extern "C" int pe_oracle_eval(int32_t V, int32_t E, const int32_t* edge_src, const int32_t* edge_dst,
+                              const int32_t* dur, const int32_t* mem_delta, const int32_t* mem_weight, int32_t D,
+                              int32_t L, const uint8_t* link_class, const int32_t* comm,
+                              const int32_t* mem_capacity, int64_t K, int64_t c_begin, int64_t c_end,
+                              const uint8_t* assign, const void* order, int order_bytes, uint32_t flags,
+                              int32_t* start, int32_t* finish, int32_t* makespan, int32_t* busy, int32_t* peak_mem,
+                              uint32_t* status) {
+  return pe_oracle_eval_hetero(V, E, edge_src, edge_dst, dur, nullptr, mem_delta, mem_weight, D, L, link_class, comm,
+                               mem_capacity, K, c_begin, c_end, assign, order, order_bytes, flags, start, finish,
+                               makespan, busy, peak_mem, status);
 }
 
 // ---------------------------------------------------------------------------------------------

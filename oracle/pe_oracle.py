@@ -42,6 +42,10 @@ def _load():
         lib.pe_oracle_eval.argtypes = [ctypes.c_int32, ctypes.c_int32, P, P, P, P, P, ctypes.c_int32, ctypes.c_int32,
                                        P, P, P, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, P, P, ctypes.c_int,
                                        ctypes.c_uint32, P, P, P, P, P, P]
+        lib.pe_oracle_eval_hetero.restype = ctypes.c_int
+        lib.pe_oracle_eval_hetero.argtypes = [ctypes.c_int32, ctypes.c_int32, P, P, P, P, P, P, ctypes.c_int32,
+                                              ctypes.c_int32, P, P, P, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                                              P, P, ctypes.c_int, ctypes.c_uint32, P, P, P, P, P, P]
         lib.pe_oracle_decode.restype = ctypes.c_int
         lib.pe_oracle_decode.argtypes = [ctypes.c_int32, ctypes.c_int32, P, P, ctypes.c_int64, ctypes.c_int64,
                                          ctypes.c_int64, P, ctypes.c_int, P, P]
@@ -73,6 +77,8 @@ def evaluate(w, assign, order, flags=0, want_times=True, threads=1, c_range=None
     src, dst = _c(w.edge_src, np.int32), _c(w.edge_dst, np.int32)
     dur, A, W = _c(w.dur, np.int32), _c(w.mem_delta, np.int32), _c(w.mem_weight, np.int32)
     cls, comm, cap = _c(w.link_class, np.uint8), _c(w.comm, np.int32), _c(w.mem_capacity, np.int32)
+    durm = _c(getattr(w, "dur_by_machine", None), np.int32)      # [V, D]: heterogeneous machines (Section III, footnote)
+    assert durm is None or durm.shape == (V, D)
     E = int(src.shape[0])
     out = dict(
         start=np.zeros((V, K), np.int32) if want_times else None,
@@ -83,10 +89,10 @@ def evaluate(w, assign, order, flags=0, want_times=True, threads=1, c_range=None
     b, e = (0, K) if c_range is None else c_range
 
     def run(lo, hi):
-        rc = lib.pe_oracle_eval(V, E, _p(src), _p(dst), _p(dur), _p(A), _p(W), D, L, _p(cls), _p(comm), _p(cap),
-                                K, lo, hi, _p(assign), _p(order), order.dtype.itemsize, flags,
-                                _p(out["start"]), _p(out["finish"]), _p(out["makespan"]), _p(out["busy"]),
-                                _p(out["peak_mem"]), _p(out["status"]))
+        rc = lib.pe_oracle_eval_hetero(V, E, _p(src), _p(dst), _p(dur), _p(durm), _p(A), _p(W), D, L, _p(cls), _p(comm),
+                                       _p(cap), K, lo, hi, _p(assign), _p(order), order.dtype.itemsize, flags,
+                                       _p(out["start"]), _p(out["finish"]), _p(out["makespan"]), _p(out["busy"]),
+                                       _p(out["peak_mem"]), _p(out["status"]))
         if rc != 0:
             raise RuntimeError(f"pe_oracle_eval failed with code {rc}")
 
