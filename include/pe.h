@@ -65,6 +65,13 @@ typedef struct {
                                   the diagonal is ignored; 0xFF = no channel (Eq. 10); NULL = all class 0 */
   const int32_t* comm;         /* [E*L] D^c of edge e over link class l at e*L + l, >= 0; NULL = all 0 */
   const int32_t* mem_capacity; /* [D] memory limit per machine; NULL = no limit */
+  const int32_t* dur_by_machine; /* [V*D] heterogeneous machines (Section III, footnote: the model extends by giving
+                                  the duration a machine index): operator i lasts dur_by_machine[i*D + j] >= 0 on
+                                  machine j, D^o_i of Eq. 3 becoming D^o_{i,x_i}; NULL = homogeneous (`dur` applies).
+                                  `dur` must still be given (it is ignored by the evaluation when this is set).
+                                  Such graphs are evaluated by the one-thread-per-candidate kernels
+                                  (PE_VARIANT_SHARED / PE_VARIANT_GLOBAL); PE_VARIANT_WARP and PE_VARIANT_TEAM return
+                                  PE_ERR_UNSUPPORTED for them. */
 } pe_graph_desc;
 
 /* Host-only check of a description: ranges, acyclicity, overflow bounds.  Touches no GPU. */
@@ -246,7 +253,8 @@ int pe_select_best(int64_t K, const int32_t* makespan, const uint32_t* status, u
  * (NULL allowed if the input has no comm), sorted by (source, destination); dur [V]; mem_delta, mem_weight [V]
  * (each may be NULL).  Only the first *num_ops_out / *num_edges_out entries are written.  The result is a
  * DAG and can go straight into pe_graph_create.  V above 16384 is PE_ERR_UNSUPPORTED (the adjacency is kept
- * as two V x V bit matrices); the description is validated first (PE_ERR_CYCLE, PE_ERR_RANGE, ...). */
+ * as two V x V bit matrices), as is a description with dur_by_machine (Section IV sums one duration per
+ * operator); the description is validated first (PE_ERR_CYCLE, PE_ERR_RANGE, ...). */
 typedef struct {
   int32_t target_ops;      /* N >= 1: stop once |I| <= N */
   int32_t max_dur_edge;    /* thresholds of merges along an edge */

@@ -120,6 +120,25 @@ def select_best(makespan, status, reject_mask=0xFFFFFFFF):
     return best_c, best, count
 
 
+def select_topk(makespan, status, k, reject_mask=0xFFFFFFFF):
+    """The k best candidates written out (Eq. 1: smaller makespan is better; Section III: a candidate whose
+    status has a `reject_mask` bit is not a valid arrangement): repeatedly take, among the qualifying
+    candidates not yet taken, the one with the smallest makespan, ties to the smallest index.  Returns the
+    chosen indices in INCREASING INDEX order (the selection is a set; at most k, fewer if fewer qualify)."""
+    taken = []
+    for _ in range(int(k)):
+        best_c = -1
+        for c in range(len(makespan)):
+            if (int(status[c]) & reject_mask) or c in taken:
+                continue
+            if best_c < 0 or int(makespan[c]) < int(makespan[best_c]):
+                best_c = c
+        if best_c < 0:
+            break
+        taken.append(best_c)
+    return sorted(taken)
+
+
 def decode(w, plist, threads=1):
     """Priority-list decoding (see pe_oracle.cpp): plist is u16/u32 [V, K], plist[r, c] = the operation of
     rank r of candidate c.  Returns (order [V, K] of the same dtype, status [K] uint32)."""

@@ -37,7 +37,8 @@ _P = ctypes.c_void_p
 class pe_graph_desc(ctypes.Structure):
     _fields_ = [("num_ops", ctypes.c_int32), ("num_edges", ctypes.c_int32), ("edge_src", _P), ("edge_dst", _P),
                 ("dur", _P), ("mem_delta", _P), ("mem_weight", _P), ("num_devices", ctypes.c_int32),
-                ("num_link_classes", ctypes.c_int32), ("link_class", _P), ("comm", _P), ("mem_capacity", _P)]
+                ("num_link_classes", ctypes.c_int32), ("link_class", _P), ("comm", _P), ("mem_capacity", _P),
+                ("dur_by_machine", _P)]
 
 
 class pe_outputs(ctypes.Structure):
@@ -110,7 +111,7 @@ def _np_ptr(a, dtype):
 
 
 def make_desc(num_ops, edge_src, edge_dst, dur, num_devices, mem_delta=None, mem_weight=None, num_link_classes=1,
-              link_class=None, comm=None, mem_capacity=None):
+              link_class=None, comm=None, mem_capacity=None, dur_by_machine=None):
     """Fill a pe_graph_desc from numpy arrays; returns (desc, keepalive list)."""
     keep = []
     d = pe_graph_desc()
@@ -121,7 +122,7 @@ def make_desc(num_ops, edge_src, edge_dst, dur, num_devices, mem_delta=None, mem
     for name, arr, dt in (("edge_src", edge_src, np.int32), ("edge_dst", edge_dst, np.int32), ("dur", dur, np.int32),
                           ("mem_delta", mem_delta, np.int32), ("mem_weight", mem_weight, np.int32),
                           ("link_class", link_class, np.uint8), ("comm", comm, np.int32),
-                          ("mem_capacity", mem_capacity, np.int32)):
+                          ("mem_capacity", mem_capacity, np.int32), ("dur_by_machine", dur_by_machine, np.int32)):
         ptr, ka = _np_ptr(arr, dt)
         setattr(d, name, ptr)
         keep.append(ka)
@@ -131,7 +132,7 @@ def make_desc(num_ops, edge_src, edge_dst, dur, num_devices, mem_delta=None, mem
 def desc_from_workload(w):
     return make_desc(w.num_ops, w.edge_src, w.edge_dst, w.dur, w.num_devices, mem_delta=w.mem_delta,
                      mem_weight=w.mem_weight, num_link_classes=w.num_link_classes, link_class=w.link_class,
-                     comm=w.comm, mem_capacity=w.mem_capacity)
+                     comm=w.comm, mem_capacity=w.mem_capacity, dur_by_machine=getattr(w, "dur_by_machine", None))
 
 
 def pe_coarsen(desc, target_ops, max_dur_edge, max_mem_edge, max_dur_nonedge, max_mem_nonedge):

@@ -160,6 +160,7 @@ extern "C" int pe_coarsen(const pe_graph_desc* desc, const pe_coarsen_params* pr
   const int V = desc->num_ops, E = desc->num_edges, L = desc->num_link_classes;
   if (E > 0 && (!edge_src || !edge_dst)) return PE_ERR_INVALID_ARG;
   if (V > 16384) return PE_ERR_UNSUPPORTED;   // bit-matrix adjacency: 2 x V^2 / 8 bytes
+  if (desc->dur_by_machine) return PE_ERR_UNSUPPORTED;   // Section IV sums one duration per operator
   if (prm->target_ops < 1) return PE_ERR_INVALID_ARG;
   Coarsener g;
   g.V = V; g.L = L; g.words = (V + 63) / 64; g.nlive = V;

@@ -16,6 +16,7 @@ struct GraphPtrs {
   const int32_t* weight;  // nullptr when the graph has no W
   const uint8_t* cls;
   const int32_t* cap;
+  const int32_t* durm;    // nullptr unless durations depend on the machine
 };
 
 __device__ __forceinline__ GraphPtrs graph_ptrs(const uint8_t* base, const PeGraphView& g) {
@@ -26,6 +27,7 @@ __device__ __forceinline__ GraphPtrs graph_ptrs(const uint8_t* base, const PeGra
   p.weight = g.has_weight ? reinterpret_cast<const int32_t*>(base + g.lay.weight) : nullptr;
   p.cls = base + g.lay.cls;
   p.cap = reinterpret_cast<const int32_t*>(base + g.lay.cap);
+  p.durm = g.hetero ? reinterpret_cast<const int32_t*>(base + g.lay.durm) : nullptr;
   return p;
 }
 

@@ -100,12 +100,13 @@ __global__ void pe_eval_global_kernel(PeGraphView g, const uint8_t* __restrict__
       }
       r = max(r, ep);
     }
+    const int32_t d_i = gp.durm ? gp.durm[(size_t)i * D + j] : op.dur;   // D^o of i on its machine (Eq. 3)
     const int32_t s = max(r, free_at[j * T]);
-    const int32_t e = s + op.dur;
+    const int32_t e = s + d_i;
     free_at[j * T] = e;
     e_state[(size_t)i * Ks + c] = e;
     if (BY_POS) x_state[(size_t)i * Ks + c] = (uint8_t)j;
-    busy[j * T] += op.dur;
+    busy[j * T] += d_i;
     const int32_t lv = lvl[j * T] + op.mem_delta;
     lvl[j * T] = lv;
     peak[j * T] = max(peak[j * T], lv);
@@ -199,11 +200,12 @@ __global__ void pe_eval_shared_kernel(PeGraphView g, const uint8_t* __restrict__
       }
       r = max(r, ep);
     }
+    const int32_t d_i = gp.durm ? gp.durm[(size_t)i * D + j] : op.dur;   // D^o of i on its machine (Eq. 3)
     const int32_t s = max(r, free_at[j * T]);
-    const int32_t e = s + op.dur;
+    const int32_t e = s + d_i;
     free_at[j * T] = e;
     state[(size_t)i * T] = pack_state((uint32_t)e, (uint32_t)j);
-    busy[j * T] += op.dur;
+    busy[j * T] += d_i;
     const int32_t lv = lvl[j * T] + op.mem_delta;
     lvl[j * T] = lv;
     peak[j * T] = max(peak[j * T], lv);
@@ -406,6 +408,14 @@ static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, bool allow_co
   if (flags & ~(uint32_t)(PE_ASSIGN_BY_POS | PE_TIMES_BY_OP | PE_COMM_EXCLUSIVE | PE_VARIANT_MASK)) return PE_ERR_INVALID_ARG;
   *p = Plan();
   const uint32_t want = flags & PE_VARIANT_MASK;
+  if (g->hetero) {   // machine-dependent durations: the generic one-thread-per-candidate kernels
+    if (want == PE_VARIANT_WARP || want == PE_VARIANT_TEAM) return PE_ERR_UNSUPPORTED;
+    if (!(flags & PE_COMM_EXCLUSIVE) && want != PE_VARIANT_GLOBAL && plan_shared(g, false, p) &&
+        (p->threads >= 48 || want == PE_VARIANT_SHARED))
+      return PE_OK;
+    if (want == PE_VARIANT_SHARED) return PE_ERR_UNSUPPORTED;
+    return plan_global(g, K, flags, false, p) ? PE_OK : PE_ERR_UNSUPPORTED;
+  }
   if (flags & PE_COMM_EXCLUSIVE) {
     // exclusive channels: the compact shared-state kernel where a block of candidates still fits with one
     // more word per machine pair each, else the generic global-state kernel

@@ -23,7 +23,16 @@ int check_desc(const pe_graph_desc* d, int64_t* time_bound, int64_t* mem_bound, 
   int64_t tsum = 0, msum = 0;
   for (int32_t i = 0; i < V; ++i) {
     if (d->dur[i] < 0) return PE_ERR_RANGE;
-    tsum += d->dur[i];
+    int64_t longest = d->dur[i];
+    if (d->dur_by_machine) {   // heterogeneous machines: the bound takes the slowest machine
+      longest = 0;
+      for (int32_t j = 0; j < D; ++j) {
+        const int32_t t = d->dur_by_machine[(size_t)i * D + j];
+        if (t < 0) return PE_ERR_RANGE;
+        if (t > longest) longest = t;
+      }
+    }
+    tsum += longest;
     if (d->mem_delta) msum += d->mem_delta[i] < 0 ? -(int64_t)d->mem_delta[i] : (int64_t)d->mem_delta[i];
     if (d->mem_weight) {
       if (d->mem_weight[i] < 0) return PE_ERR_RANGE;
@@ -96,6 +105,7 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
   g->V = V; g->E = E; g->D = D; g->L = L;
   g->device = cuda_device;
   g->has_weight = d->mem_weight != nullptr;
+  g->hetero = d->dur_by_machine != nullptr;
   g->time_bound = tb; g->mem_bound = mb; g->max_indeg = mdeg;
   g->d_blob = nullptr; g->d_error = nullptr;
 
@@ -107,6 +117,7 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
   lay.weight = (uint32_t)at; at = align16(at + (g->has_weight ? (uint64_t)V * 4 : 0));
   lay.cls = (uint32_t)at;    at = align16(at + (uint64_t)D * D);
   lay.cap = (uint32_t)at;    at = align16(at + (uint64_t)D * 4);
+  lay.durm = (uint32_t)at;   at = align16(at + (g->hetero ? (uint64_t)V * D * 4 : 0));
   if (at > 0x7FFFFFF0ull) { delete g; return PE_ERR_INVALID_ARG; }
   lay.bytes = (uint32_t)at;
 
@@ -134,6 +145,7 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
   }
   if (g->has_weight) std::memcpy(blob.data() + lay.weight, d->mem_weight, (size_t)V * 4);
   if (d->link_class) std::memcpy(blob.data() + lay.cls, d->link_class, (size_t)D * D);
+  if (g->hetero) std::memcpy(blob.data() + lay.durm, d->dur_by_machine, (size_t)V * D * 4);
   int32_t* cap = (int32_t*)(blob.data() + lay.cap);
   for (int32_t j = 0; j < D; ++j) cap[j] = d->mem_capacity ? d->mem_capacity[j] : INT32_MAX;
 
@@ -141,7 +153,7 @@ extern "C" int pe_graph_create(const pe_graph_desc* d, int cuda_device, pe_graph
   bool no_channel = false;
   if (d->link_class)
     for (int32_t a = 0; a < D * D; ++a) no_channel = no_channel || d->link_class[a] == 0xFF;
-  bool narrow = V <= 65535 && L <= 2 && mdeg <= 255 && E < (1 << 24);
+  bool narrow = V <= 65535 && L <= 2 && mdeg <= 255 && E < (1 << 24) && !g->hetero;   // (the compact record has one duration)
   for (int32_t i = 0; narrow && i < V; ++i)
     narrow = ops[i].dur <= 65535 && ops[i].mem_delta >= -128 && ops[i].mem_delta <= 127;
   for (int64_t q = 0; narrow && q < (int64_t)E * L; ++q) narrow = comm[q] <= 65535;

@@ -26,6 +26,7 @@ struct PeBlobLayout {
   uint32_t weight;  // int32[V]      W_i (present only if has_weight)
   uint32_t cls;     // uint8[D*D]    link class of (machine of predecessor, machine of successor)
   uint32_t cap;     // int32[D]      capacity (INT32_MAX where there is no limit)
+  uint32_t durm;    // int32[V*D]    duration of operator i on machine j at i*D + j (present only if hetero)
   uint32_t bytes;   // total, multiple of 16
 };
 
@@ -33,6 +34,7 @@ struct PeBlobLayout {
 struct PeGraphView {
   int32_t V, E, D, L;
   int32_t has_weight;
+  int32_t hetero;   // durations depend on the machine (the blob holds durm)
   PeBlobLayout lay;
 };
 
@@ -75,6 +77,7 @@ struct pe_graph {
   int32_t V, E, D, L;
   int device;
   bool has_weight;
+  bool hetero;         // durations depend on the machine
   int64_t time_bound;  // sum dur + sum_e max_l comm: no start/end time exceeds it
   int64_t mem_bound;   // sum |A| + sum W
   int32_t max_indeg;
@@ -109,6 +112,7 @@ inline PeGraphView pe_view(const pe_graph* g) {
   PeGraphView v;
   v.V = g->V; v.E = g->E; v.D = g->D; v.L = g->L;
   v.has_weight = g->has_weight ? 1 : 0;
+  v.hetero = g->hetero ? 1 : 0;
   v.lay = g->lay;
   return v;
 }

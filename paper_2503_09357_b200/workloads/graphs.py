@@ -107,6 +107,28 @@ def bidirectional_pipeline(P: int = 8, M: int = 20, K: int = 65536, seed: int = 
         assign_mode="group_perm", group=_i32(ids % P), meta=dict(P=P, M=M))
 
 
+def bidirectional_unit(PP: int, M: int) -> Workload:
+    """The bidirectional pipeline at the unit times of the paper's first experiment (Section V-A):
+    T_f = T_i = T_w = 1 (forward, backward-for-input, backward-for-weights; a full backward is
+    T_b = T_i + T_w = 2), stages = machines = PP, no communication time, and the memory limit
+    "2 x parameters + (PP + 1) activations": every machine holds the parameters of its slot for both
+    directions (W = 1 on one forward operator per slot and direction), an activation (A = +1) lives from a
+    microbatch's forward operator to its weight-gradient operator (A = -1), capacity 2 + PP + 1.
+    Same operator numbering and edges as `bidirectional_pipeline`; slot p belongs on machine p.
+    The paper does not print its microbatch count, so M is the caller's choice."""
+    w = bidirectional_pipeline(P=PP, M=M, K=1)
+    V = w.num_ops
+    ids = np.arange(V)
+    kind, m_of = ids // (M * PP), (ids // PP) % M
+    w.name = f"bidirectional_unit_PP{PP}_M{M}"
+    w.dur = _i32(np.ones(V))
+    w.comm = _i32(np.zeros_like(w.comm))
+    w.mem_delta = _i32(np.where(kind == 0, 1, np.where(kind == 2, -1, 0)))
+    w.mem_weight = _i32((kind == 0) & ((m_of == 0) | (m_of == M // 2)))
+    w.mem_capacity = _i32(np.full(PP, 2 + PP + 1))
+    return w
+
+
 def _two_class_comm(seed, E):
     nbytes = rng.randint(seed, _S_COMM, np.arange(E), 0, 1, 64)
     return _i32(np.stack([(nbytes + 3) // 4, nbytes], axis=1))   # intra-node bw 4, inter-node bw 1

@@ -358,3 +358,21 @@ def test_select_best_hand_cases():
     assert orc.select_best([5, 3], [2, 1]) == (-1, 2 ** 31 - 1, 0)
     assert orc.select_best([], []) == (-1, 2 ** 31 - 1, 0)
     assert orc.select_best([7], [8], reject_mask=4) == (0, 7, 1)
+
+
+def test_select_topk_hand_cases_and_library_sort():
+    mk = [9, 4, 7, 4, 4, 12, 1]
+    st = [0, 0, 2, 0, 4, 0, 1]
+    assert orc.select_topk(mk, st, 3) == [0, 1, 3]                    # 4 (c=1), 4 (c=3), then 9; status != 0 never
+    assert orc.select_topk(mk, st, 1) == [1]                          # ties go to the smallest index
+    assert orc.select_topk(mk, st, 3, reject_mask=3) == [1, 3, 4]     # bit 4 tolerated: three 4s
+    assert orc.select_topk(mk, st, 10) == [0, 1, 3, 5]                # fewer qualify than asked for
+    assert orc.select_topk(mk, st, 0) == [] and orc.select_topk([], [], 3) == []
+    assert orc.select_topk(mk, st, 1) == [orc.select_best(mk, st)[0]]
+    rs = np.random.RandomState(11)
+    for _ in range(20):                                               # against numpy's stable sort of (makespan, index)
+        n = int(rs.randint(1, 60)); k = int(rs.randint(0, n + 3))
+        mk = rs.randint(0, 8, n); st = rs.randint(0, 2, n) * rs.randint(1, 16, n)
+        ok = np.flatnonzero(st == 0)
+        want = sorted(ok[np.argsort(mk[ok], kind="stable")][:k].tolist())
+        assert orc.select_topk(mk, st, k) == want

@@ -43,3 +43,40 @@ def test_search_finds_the_pipeline_optimum_and_reports_what_the_oracle_computes(
         assert int(ref2["makespan"][0]) == 72 and int(ref2["status"][0]) == 0
     finally:
         g.close()
+
+
+def test_search_reaches_the_zero_bubble_of_the_two_stage_bidirectional_pipeline():
+    """Section V-A at the paper's unit times: for PP = 2 the bubble of the bidirectional pipeline is 0
+    (tests/golden/bidirectional_pp2_zero_bubble.txt pins that value on the oracle).  The search has to find
+    it from random priority lists, within the memory limit 2 x parameters + (PP + 1) activations; the PP = 4
+    run is reported as context only (the paper's microbatch count is not printed)."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    from oracle import pe_oracle as orc
+    from paper_2503_09357_b200 import binding as pe
+    from paper_2503_09357_b200 import search
+    from paper_2503_09357_b200.workloads import graphs
+    for PP, M, must in ((2, 4, 0), (4, 8, None)):
+        w = graphs.bidirectional_unit(PP, M)
+        V, K = w.num_ops, 8192
+        slot = (np.arange(V) % PP).astype(np.uint8)                          # slot p on machine p
+        assign = torch.from_numpy(np.repeat(slot[:, None], K, axis=1).copy()).cuda()
+        gen = torch.Generator(device="cuda"); gen.manual_seed(PP * 100 + M)
+        lists = torch.argsort(torch.rand((V, K), device="cuda", generator=gen), dim=0).to(torch.int16).contiguous()
+        g = pe.Graph(w)
+        try:
+            res = search.evolve(g, assign, lists, generations=150, swaps=2, seed=3)
+            busy = 3 * M                                                     # F + B + W of every microbatch, one unit each
+            bubble = res["best_makespan"] - busy
+            ref = orc.evaluate(w, res["best_assign"].cpu().numpy()[:, None],
+                               res["best_order"].cpu().numpy().view(np.uint16)[:, None])
+            assert int(ref["makespan"][0]) == res["best_makespan"] and int(ref["status"][0]) == 0
+            assert (ref["busy"][:, 0] == busy).all() and (ref["peak_mem"][:, 0] <= 2 + PP + 1).all()
+            assert bubble >= 0
+            if must is not None:
+                assert bubble == must
+            print(f"bidirectional unit pipeline PP={PP} M={M}: bubble {bubble} "
+                  f"(Section V-A: best found PP/2-1 = {PP // 2 - 1}, DualPipe 2(PP/2-1) = {2 * (PP // 2 - 1)})")
+        finally:
+            g.close()
