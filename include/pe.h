@@ -228,6 +228,20 @@ int pe_decode_priority(pe_graph* g, int64_t K, const void* list, int order_bytes
 int pe_select_best(int64_t K, const int32_t* makespan, const uint32_t* status, uint32_t reject_mask, int64_t* result,
                    void* cuda_stream);
 
+/* The k best candidates of an evaluation (Eq. 1; Section III validity as for pe_select_best): the qualifying
+ * candidates (status has none of the `reject_mask` bits) with the smallest makespans, ties to the smallest
+ * candidate index - what a search keeps as its elite.  The selection is a set: out_index lists it by
+ * INCREASING CANDIDATE INDEX, not by makespan.
+ *   makespan, status   device, [K], as written by pe_eval_batch
+ *   k                  how many to keep (>= 0)
+ *   out_index          device, int32 [k]: the chosen candidates; entries beyond *out_count are -1
+ *   out_count          device, one int32: min(k, number of qualifying candidates)
+ *   workspace          device scratch of at least pe_select_topk_workspace_bytes(K) bytes, 16-byte aligned
+ * Asynchronous on `cuda_stream`; runs on the device that owns out_count.  K must be below 2^31. */
+size_t pe_select_topk_workspace_bytes(int64_t K);
+int pe_select_topk(int64_t K, const int32_t* makespan, const uint32_t* status, uint32_t reject_mask, int32_t k,
+                   int32_t* out_index, int32_t* out_count, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Operator merging in front of candidate generation (Section IV, Algorithm 1): shrinks G_m(I, B) to at most
  * `target_ops` operators by repeatedly merging pairs, so that a search (or the paper's MIP) works on a graph
  * of manageable size.  Host-only: every pointer is a HOST pointer and no GPU is touched.

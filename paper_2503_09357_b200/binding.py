@@ -73,6 +73,10 @@ _lib.pe_decode_priority.restype = ctypes.c_int
 _lib.pe_decode_priority.argtypes = [_P, ctypes.c_int64, _P, ctypes.c_int, ctypes.c_uint32, _P, _P, _P, ctypes.c_size_t, _P]
 _lib.pe_select_best.restype = ctypes.c_int
 _lib.pe_select_best.argtypes = [ctypes.c_int64, _P, _P, ctypes.c_uint32, _P, _P]
+_lib.pe_select_topk_workspace_bytes.restype = ctypes.c_size_t
+_lib.pe_select_topk_workspace_bytes.argtypes = [ctypes.c_int64]
+_lib.pe_select_topk.restype = ctypes.c_int
+_lib.pe_select_topk.argtypes = [ctypes.c_int64, _P, _P, ctypes.c_uint32, ctypes.c_int32, _P, _P, _P, ctypes.c_size_t, _P]
 _lib.pe_graph_poll_error.restype = ctypes.c_int
 _lib.pe_graph_poll_error.argtypes = [_P, _P]
 _lib.pe_selftest_wait_timeout.restype = ctypes.c_int
@@ -215,6 +219,16 @@ def pe_select_best(K, makespan_ptr, status_ptr, reject_mask, result_ptr, stream=
                                result_ptr, stream or None)
 
 
+def pe_select_topk_workspace_bytes(K: int) -> int:
+    return int(_lib.pe_select_topk_workspace_bytes(int(K)))
+
+
+def pe_select_topk(K, makespan_ptr, status_ptr, reject_mask, k, out_index_ptr, out_count_ptr, workspace_ptr,
+                   workspace_bytes, stream=0) -> int:
+    return _lib.pe_select_topk(int(K), makespan_ptr, status_ptr, int(reject_mask) & 0xFFFFFFFF, int(k), out_index_ptr,
+                               out_count_ptr, workspace_ptr, int(workspace_bytes), stream)
+
+
 def pe_decode_workspace_bytes(handle, K: int, flags: int = 0) -> int:
     return int(_lib.pe_decode_workspace_bytes(handle, int(K), int(flags)))
 
@@ -296,6 +310,25 @@ class Graph:
             raise PeError(rc, "pe_select_best")
         idx, mk, cnt, _ = res.tolist()
         return idx, mk, cnt
+
+    def select_topk(self, out, k, reject_mask=0xFFFFFFFF, stream=None):
+        """The k best qualifying candidates of an eval_batch result: (indices int32 [k] on the device, listed by
+        increasing candidate index and padded with -1; count, a one-element int32 device tensor).  Asynchronous."""
+        import torch
+        K = out["makespan"].numel()
+        dev = out["makespan"].device
+        idx = torch.empty(max(int(k), 1), dtype=torch.int32, device=dev)
+        cnt = torch.empty(1, dtype=torch.int32, device=dev)
+        n = pe_select_topk_workspace_bytes(K)
+        ws = torch.empty(n, dtype=torch.uint8, device=dev)
+        s = torch.cuda.current_stream(self.device).cuda_stream if stream is None else stream
+        rc = pe_select_topk(K, out["makespan"].data_ptr(), out["status"].data_ptr(), reject_mask, k, idx.data_ptr(),
+                            cnt.data_ptr(), ws.data_ptr(), n, s)
+        if rc != PE_OK:
+            raise PeError(rc, "pe_select_topk")
+        if stream is not None:
+            ws.record_stream(torch.cuda.ExternalStream(stream, device=dev))
+        return idx[:int(k)], cnt
 
     def decode_priority(self, plist, flags=0, stream=None):
         """plist: cuda int16 [V, K] holding u16 operator ids, plist[r, c] = operator of rank r of candidate c.

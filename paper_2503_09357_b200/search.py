@@ -15,10 +15,25 @@ the three entry points working together on the device; it is not part of the eva
 `evolve` mutates lists and assignments directly; `evolve_keys` is the biased random-key variant for fixed
 assignments (a candidate is a vector of keys, its priority list their argsort).
 
-torch is used for the mutations (gather/scatter on the device) and for picking survivors;
-the scheduling arithmetic is all in the library's kernels.
+torch is used for the mutations (gather/scatter on the device) only; decoding, the scheduling arithmetic
+and the choice of the survivors (pe_select_topk, pe_select_best) are all in the library's kernels.
 """
 import numpy as np
+
+
+def _elite(graph, out, n, reject_mask):
+    """The elite of a generation through the library's selection steps: the n best qualifying candidates
+    (pe_select_topk; padded by repeating the first one when fewer qualify, or by candidate 0 when none does)
+    and the best of all (pe_select_best).  Returns (elite indices [n], how many qualify, best index, its
+    makespan or INT32_MAX)."""
+    import torch
+    idx, cnt = graph.select_topk(out, n, reject_mask)
+    c, mk, _ = graph.select_best(out, reject_mask)
+    n_ok = int(cnt.item())
+    idx = idx.to(torch.int64)
+    if n_ok < n:
+        idx = torch.where(torch.arange(n, device=idx.device) < n_ok, idx, idx[0].clamp(min=0))
+    return idx, n_ok, max(c, 0), (mk if c >= 0 else torch.iinfo(torch.int32).max)
 
 
 def evolve(graph, assign, lists, generations=20, elite=0.125, swaps=2, reassign=0, num_devices=None, seed=0,
@@ -37,13 +52,10 @@ def evolve(graph, assign, lists, generations=20, elite=0.125, swaps=2, reassign=
     for _ in range(generations):
         order, dstatus = graph.decode_priority(lists)
         out = graph.eval_batch(assign, order, flags=flags, want_times=False)
-        bad = ((out["status"] & np.int32(np.uint32(reject_mask).view(np.int32))) != 0) | (dstatus != 0)
-        score = torch.where(bad, torch.full_like(out["makespan"], big), out["makespan"])
-        top = torch.argsort(score, stable=True)[:n_elite]
-        gbest = int(score[top[0]])
+        out["status"] |= dstatus                               # a list that is not a permutation is no candidate
+        top, n_ok, c, gbest = _elite(graph, out, n_elite, reject_mask)
         best["history"].append(gbest)
         if gbest < best["best_makespan"]:
-            c = int(top[0])
             best.update(best_makespan=gbest, best_assign=assign[:, c].clone(), best_list=lists[:, c].clone(),
                         best_order=order[:, c].clone())
         # next generation: the elite unchanged, the rest mutated copies of random elite members
@@ -88,13 +100,11 @@ def evolve_keys(graph, assign, generations=200, elite=0.1, mutants=0.2, bias=0.7
         lists = torch.argsort(keys, dim=0).to(torch.int16).contiguous()
         order, dstatus = graph.decode_priority(lists)
         out = graph.eval_batch(assign, order, flags=flags, want_times=False)
-        bad = ((out["status"] & mask_bits) != 0) | (dstatus != 0)
-        score = torch.where(bad, torch.full_like(out["makespan"], big), out["makespan"])
-        top = torch.argsort(score, stable=True)[:n_el]
-        gbest = int(score[top[0]])
+        out["status"] |= dstatus
+        top, n_ok, c, gbest = _elite(graph, out, n_el, reject_mask)
         best["history"].append(gbest)
         if gbest < best["best_makespan"]:
-            best.update(best_makespan=gbest, best_order=order[:, top[0]].clone(), best_column=int(top[0]))
+            best.update(best_makespan=gbest, best_order=order[:, c].clone(), best_column=c)
         pa = top[torch.randint(0, n_el, (K,), device=dev, generator=gen)]
         pb = torch.randint(0, K, (K,), device=dev, generator=gen)
         take = torch.rand((V, K), device=dev, generator=gen) < bias

@@ -391,3 +391,34 @@ def test_other_sweep_points_at_full_size_sampled(pe, V, D):
         assert bool((out["makespan"].view(K // base, base) == first).all())       # every repeat like its original
     finally:
         g.close()
+
+
+def test_select_topk_matches_the_definition(pe):
+    """pe_select_topk against its definition written out in the oracle (small K) and, at sizes where that loop
+    is too slow, against numpy's stable sort of (makespan, index), which the oracle's pins show to be the same."""
+    import torch
+    from oracle import pe_oracle as orc
+    w = wl.make_config(1)
+    g = pe.Graph(w)
+    try:
+        rs = np.random.RandomState(7)
+        for K, k, hi in ((1, 1, 5), (37, 5, 3), (1000, 100, 50), (4097, 4097, 9), (5000, 0, 10), (3000, 4000, 10 ** 6),
+                         (300000, 30000, 1 << 20), (300000, 1000, 40)):
+            mk = rs.randint(0, hi, K).astype(np.int32)
+            st = (rs.randint(0, 4, K) == 0).astype(np.uint32) * rs.randint(1, 16, K).astype(np.uint32)
+            if K == 4097:
+                mk[:] = 7                                        # all equal: the choice is by index alone
+            out = dict(makespan=torch.from_numpy(mk).cuda(), status=torch.from_numpy(st.view(np.int32)).cuda())
+            for mask in (0xFFFFFFFF, 3):
+                idx, cnt = g.select_topk(out, k, mask)
+                torch.cuda.synchronize()
+                idx, cnt = idx.cpu().numpy(), int(cnt.item())
+                ok = np.flatnonzero((st & np.uint32(mask)) == 0)
+                want = sorted(ok[np.argsort(mk[ok], kind="stable")][:k].tolist())
+                if K <= 1000:
+                    assert want == orc.select_topk(mk, st, k, mask)
+                assert cnt == len(want), (K, k, mask)
+                assert idx[:cnt].tolist() == want, (K, k, mask)
+                assert (idx[cnt:] == -1).all()
+    finally:
+        g.close()
