@@ -359,7 +359,7 @@ def test_bounded_wait_reports_a_timeout_and_leaves_the_graph_usable(pe):
         g.close()
 
 
-@pytest.mark.parametrize("V,D", [(256, 64), (1024, 8), (1024, 64), (4096, 8)])
+@pytest.mark.parametrize("V,D", [(256, 8), (256, 64), (1024, 8), (1024, 64), (4096, 8), (4096, 64), (16384, 8)])
 def test_other_sweep_points_at_full_size_sampled(pe, V, D):
     """Sweep points at their full K (K * V = 2^30), i.e. in the launch shapes the benchmark times them in (ragged
     shared-state blocks at V = 1024 / D = 8, slab mode of the warp kernel at V = 1024 / D = 64, register slots with
@@ -420,5 +420,76 @@ def test_select_topk_matches_the_definition(pe):
                 assert cnt == len(want), (K, k, mask)
                 assert idx[:cnt].tolist() == want, (K, k, mask)
                 assert (idx[cnt:] == -1).all()
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("V,variant", [(256, "shared"), (256, "global"), (4096, "warp")])
+def test_batches_beyond_32_bit_element_offsets(pe, V, variant):
+    """K * V just above 2^32: the thread-per-candidate and warp-per-candidate kernels switch to 64-bit element
+    offsets there.  The batch is built on the device by repeating 8192 generated candidates; summary outputs
+    only (the times would be 34 GB); sampled columns against the oracle, every column against its twin."""
+    import torch
+    from oracle import pe_oracle as orc
+    w = wl.make_config(5, V=V, D=8)
+    base = 8192
+    reps = (1 << 32) // (V * base) + 1
+    K = base * reps
+    assert V * K > (1 << 32)
+    a0, o0 = wl.make_candidates(w, K=base)
+    flags = {"shared": pe.PE_VARIANT_SHARED, "global": pe.PE_VARIANT_GLOBAL, "warp": pe.PE_VARIANT_WARP}[variant]
+    g = pe.Graph(w)
+    try:
+        assert g.variant(K, flags) == variant
+        a = torch.from_numpy(a0).cuda().repeat(1, reps).contiguous()
+        o = torch.from_numpy(gu.as_signed(o0)).cuda().repeat(1, reps).contiguous()
+        out = g.eval_batch(a, o, flags=flags, want_times=False)
+        torch.cuda.synchronize()
+        del a, o
+        rs = np.random.RandomState(V)
+        sample = np.sort(np.concatenate([rs.choice(K, 200, replace=False), np.arange(K - 56, K)]))   # the far end too
+        st = torch.from_numpy(sample).cuda()
+        sub = {k: (v[st] if v.dim() == 1 else v[:, st]).cpu().numpy() for k, v in out.items()}
+        sub["status"] = sub["status"].view(np.uint32)
+        ref = orc.evaluate(w, np.ascontiguousarray(a0[:, sample % base]), np.ascontiguousarray(o0[:, sample % base]),
+                           want_times=False, threads=gu.CPU_THREADS)
+        gu.compare(sub, ref, f"64-bit offsets V={V} {variant}")
+        assert int(out["status"].abs().max()) == 0
+        assert bool((out["makespan"].view(reps, base) == out["makespan"][:base]).all())
+        assert bool((out["busy"].view(-1, reps, base) == out["busy"][:, :base].unsqueeze(1)).all())
+        assert bool((out["peak_mem"].view(-1, reps, base) == out["peak_mem"][:, :base].unsqueeze(1)).all())
+    finally:
+        g.close()
+        torch.cuda.empty_cache()
+
+
+def test_many_sources_of_one_operator_inside_its_window(pe):
+    """Operators with five to eight incoming edges whose sources all sit in the same 32-position window, two
+    link classes: the warp kernel then has to go back to the edge list for the sources beyond its inline
+    slots.  Orders: the identity (sources right in front of their sink) and random topological ones."""
+    rs = np.random.RandomState(42)
+    V, D, L = 96, 5, 2
+    edges = []
+    for sink, fan in ((8, 8), (20, 6), (29, 5), (40, 7), (70, 8)):
+        edges += [(sink - 1 - q, sink) for q in range(fan)]            # sources sink-fan .. sink-1
+    edges += [(i, i + 1) for i in range(0, V - 1, 3)]                  # some chains across windows
+    edges += [(int(a), int(b)) for a, b in zip(rs.randint(0, 40, 30), rs.randint(41, V, 30))]
+    edges = sorted(set(edges))
+    cls = rs.randint(0, L, (D, D)).astype(np.uint8)
+    w = ck.problem(V, edges, rs.randint(1, 20, V), D, comm=rs.randint(0, 9, (len(edges), L)), L=L, link_class=cls,
+                   A=rs.randint(-3, 4, V), cap=rs.randint(5, 30, D))
+    w.assign_mode, w.group = "per_op", None
+    K = 256
+    assign, order = wl.make_candidates(w, K=K)
+    order[:, :K // 2] = np.arange(V, dtype=order.dtype)[:, None]       # identity order for half of them
+    g = pe.Graph(w)
+    try:
+        names = []
+        for name, flags in variants_for(pe, g, K):
+            gu.check(g, w, assign, order, flags=flags, label=f"many in-window sources {name}")
+            names.append(name)
+        assert "warp" in names
+        a_pos = wl.assign_by_pos(assign, order)
+        gu.check(g, w, a_pos, order, flags=pe.PE_VARIANT_WARP | pe.PE_ASSIGN_BY_POS, label="many in-window sources by-pos")
     finally:
         g.close()

@@ -63,3 +63,60 @@ def test_noalloc_entry_point_matches_pe_eval_batch_on_two_calls_in_a_row():
         assert pe.pe_eval_batch_noalloc(g.handle, 0, 0, 0, 2, 0, pe.make_outputs(), stream) == pe.PE_OK
     finally:
         g.close()
+
+
+@pytest.mark.parametrize("case", ["generic kernel, 32-bit orders, by-position assignments", "many machines: records in the scratch too",
+                                  "start times only"])
+def test_noalloc_other_branches_of_the_scratch_layout(case):
+    """The entry point keeps different things in its built-in array depending on the problem: the generic
+    kernel's end times and machine ids, the compact kernel's per-machine records when there are many machines.
+    Each layout runs twice in a row on different candidates (the second call meets the first one's leftovers)
+    and must match both pe_eval_batch and the oracle."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    from oracle import pe_oracle as orc
+    from paper_2503_09357_b200 import binding as pe
+    if case.startswith("generic"):
+        w, ob, flags, K = wl.make_config(5, V=256, D=8), 4, pe.PE_ASSIGN_BY_POS, 1500
+    elif case.startswith("many"):
+        w, ob, flags, K = wl.make_config(5, V=256, D=64), 2, 0, 1500
+    else:
+        w, ob, flags, K = wl.make_config(1), 2, pe.PE_TIMES_BY_OP, 777
+    V = w.num_ops
+    g = pe.Graph(w)
+    try:
+        stream = torch.cuda.current_stream().cuda_stream
+        for call in range(2):
+            assign, order = wl.make_candidates(w, K=K, first=call * K, order_bytes=ob)
+            if flags & pe.PE_ASSIGN_BY_POS:
+                assign = wl.assign_by_pos(assign, order)
+            a = torch.from_numpy(assign).cuda()
+            o = torch.from_numpy(_as_signed(order)).cuda()
+            got = g.alloc_outputs(K)
+            for t in got.values():
+                t.fill_(-7)
+            ptrs = {k: v.data_ptr() for k, v in got.items()}
+            if case.startswith("start"):
+                ptrs.pop("finish")
+            rc = pe.pe_eval_batch_noalloc(g.handle, K, a.data_ptr(), o.data_ptr(), ob, flags, pe.make_outputs(**ptrs), stream)
+            assert rc == pe.PE_OK, pe.pe_strerror(rc)
+            ref = g.eval_batch(a, o, flags=flags)
+            torch.cuda.synchronize()
+            cpu = orc.evaluate(w, assign, order, flags=flags & 7, threads=8)
+            for key in ref:
+                if key == "finish" and case.startswith("start"):
+                    assert bool((got[key] == -7).all())                        # not asked for: not written
+                    continue
+                assert torch.equal(ref[key], got[key]), f"{case}, call {call}: {key} differs from pe_eval_batch"
+                want = cpu[key].view(np.int32) if key == "status" else cpu[key]
+                assert np.array_equal(got[key].cpu().numpy(), want), f"{case}, call {call}: {key} differs from the oracle"
+        if case.startswith("generic"):
+            # by-position assignments need one more byte per operator and candidate: 5 * V * K in all
+            too_many = pe.PE_NOALLOC_SCRATCH_BYTES // (5 * V) + 64
+            fits_without = pe.PE_NOALLOC_SCRATCH_BYTES // (4 * V) - 64 > too_many
+            rc = pe.pe_eval_batch_noalloc(g.handle, too_many, a.data_ptr(), o.data_ptr(), ob, flags,
+                                          pe.make_outputs(**ptrs), stream)
+            assert rc == pe.PE_ERR_SCRATCH_LIMIT and fits_without
+    finally:
+        g.close()
