@@ -40,25 +40,27 @@ FALLBACK_HBM_GBS = 6650.0
 KERNEL_OF_VARIANT = {"shared": "pe_eval_lane_kernel<STATE_SMEM=true>", "global": "pe_eval_lane_kernel<STATE_SMEM=false>",
                      "warp": "pe_eval_warp2_kernel", "team": "pe_eval_team_kernel"}
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per operator-evaluation of the
-# evaluation kernel from an ncu capture, keyed by kernel variant, valid only for the kernel
-# source whose hash is recorded with it.  Reported as null when the source has changed.
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per operator-evaluation of the evaluation kernel
+# from an ncu capture, keyed by kernel variant, valid only while the sources that kernel is built from hash to
+# the value recorded with it.  Reported as null when those sources have changed since the capture.
+KERNEL_SOURCES = {
+    "team": ("pe_kernel_team.cuh", "pe_team.cu", "pe_transpose.cuh"),
+    "warp": ("pe_kernel_warp2.cuh", "pe_warp2.cu", "pe_device.cuh", "pe_kernel_lane.cuh"),
+    "global": ("pe_kernel_lane.cuh", "pe_lane.cu", "pe_device.cuh"),
+    "shared": ("pe_kernel_lane.cuh", "pe_lane.cu", "pe_device.cuh"),
+}
 NCU_TRAFFIC = {
-    # variant: (hash of csrc/ at capture time, DRAM bytes per operator-evaluation, captured workload)
-    "global": ("0422252154d12689", 370.0, "random_layered_V16384_D64 at K = 32768 (half size), scaled by operator-evaluations"),
-    "warp": ("b3a5686239e56cfa", 10.59, "random_layered_V16384_D64 at K = 4096, scaled by operator-evaluations"),
+    # variant: (hash of its sources at capture time, DRAM bytes per operator-evaluation, captured workload)
+    "team": ("98d723e3e28e9b3f", 10.18, "random_layered_V16384_D64 at K = 3552 (one chunk), scaled by operator-evaluations; "
+                        "the staging transpositions around the kernel move another 22 B per operator-evaluation"),
 }
 
 
-EVAL_SOURCES = ("pe_device.cuh", "pe_eval.cu", "pe_graph.cu", "pe_graph.h", "pe_kernel_lane.cuh", "pe_kernel_warp.cuh",
-                "pe_kernel_warp2.cuh", "pe_kernel_team.cuh", "pe_lane.cu", "pe_launch.h", "pe_warp2.cu", "pe_team.cu")
-
-
-def kernel_source_hash():
-    """Hash of the sources the evaluation kernels are built from."""
+def kernel_source_hash(variant):
+    """Hash of the sources the kernel of `variant` is built from."""
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2503_09357_b200", "csrc")
-    for name in EVAL_SOURCES:
+    for name in KERNEL_SOURCES.get(variant, ()):
         with open(os.path.join(csrc, name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()[:16]
@@ -447,7 +449,7 @@ def run_ours(args):
         achieved = alg / (kms * 1e-3) / 1e9
         traffic = None
         rec = NCU_TRAFFIC.get(variant)
-        if rec and rec[0] == kernel_source_hash():
+        if rec and rec[0] == kernel_source_hash(variant):
             traffic = rec[1] * K * V
         cpu = None
         parity = None

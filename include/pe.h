@@ -103,7 +103,7 @@ enum {
   PE_VARIANT_WARP = 3u << 8,   /* one warp per candidate, finish-time state in shared memory */
   PE_VARIANT_TEAM = 4u << 8,   /* one block of several warps per candidate, finish-time state in shared memory; the
                                   warps prepare windows of the order side by side and only the recurrence of
-                                  Eqs. 3, 7-8, 11-13 runs window after window.  For graphs with in-degree <= 3 and
+                                  Eqs. 3, 7-8, 11-13 runs window after window.  For graphs with in-degree <= 8 and
                                   16-bit orders, with start and finish both wanted or both absent; otherwise
                                   PE_ERR_UNSUPPORTED.  Uses workspace (staging copies) when K is a multiple of 4 */
   PE_VARIANT_MASK = 15u << 8

@@ -38,6 +38,25 @@ __device__ __forceinline__ PeOpRec load_op(const PeOpRec* ops, int32_t i) {
   return r;
 }
 
+// ---- accessors over the compact encoding (PeNarrowView) ----
+struct NarrowPtrs {
+  const uint4* ops;
+  const uint32_t* edges;
+  const int32_t* weight;
+  const uint8_t* cls;
+  const int32_t* cap;
+};
+
+__device__ __forceinline__ NarrowPtrs narrow_ptrs(const uint8_t* base, const PeNarrowView& g) {
+  NarrowPtrs p;
+  p.ops = reinterpret_cast<const uint4*>(base + g.ops);
+  p.edges = reinterpret_cast<const uint32_t*>(base + g.edges);
+  p.weight = g.has_weight ? reinterpret_cast<const int32_t*>(base + g.weight) : nullptr;
+  p.cls = base + g.cls;
+  p.cap = reinterpret_cast<const int32_t*>(base + g.cap);
+  return p;
+}
+
 // ---- packed per-operator state: end time in the high 24 bits, machine in the low 8 ----
 // Used when the graph's time bound is below kPackedTimeLimit.  kNotDone marks an operator
 // that has not been scheduled yet (its machine byte is still valid).

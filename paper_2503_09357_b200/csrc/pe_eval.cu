@@ -326,7 +326,7 @@ static bool plan_warp(const pe_graph* g, int64_t K, uint32_t flags, bool allow_c
 // (the transpositions move 32-bit words) the inputs and the times go through candidate-major staging copies
 // in the workspace, a chunk of candidates at a time; a chunk is sixteen times what the GPU holds at once.
 static bool plan_team(const pe_graph* g, int64_t K, bool allow_compact, Plan* p) {
-  if (!g->narrow_ok || !allow_compact || g->max_indeg > 3 || g->time_bound >= (int64_t)1 << 23) return false;
+  if (!g->narrow_ok || !allow_compact || g->max_indeg > 8 || g->time_bound >= (int64_t)1 << 23) return false;
   const size_t smem = round_up((size_t)4 * (g->V + 2) + (size_t)4 * (5 * g->D + 2), 16);
   if (smem > g->smem_optin) return false;
   // blocks an SM holds by shared memory; six warps per block unless that would run into the SM's thread limit
@@ -443,7 +443,12 @@ static int make_plan(const pe_graph* g, int64_t K, uint32_t flags, bool allow_co
       // is faster (measured at V = 4096: 3.6e10 against 2.6e10 operator-evaluations/s at D = 64, 2.7e10
       // against 2.0e10 at D = 8; at V = 16384: 3.1e10 against 1.0e10 (warp) and 2.3e10 against 1.25e10
       // (global); at V = 1024 the single-warp kernel still wins, 4.0e10 against 3.0e10).
-      if (plan_team(g, K, allow_compact, &tm) && (!has_w || w.threads < 20 * 32)) { *p = tm; return PE_OK; }
+      // Graphs with operators of more than three incoming edges take the single-warp kernel off its register
+      // slots; there the block of warps wins as well (measured on the MoE graph: 1.7e10 against 0.9e10).
+      if (plan_team(g, K, allow_compact, &tm) && (!has_w || w.threads < 20 * 32 || (g->max_indeg > 3 && w.threads < 24 * 32))) {
+        *p = tm;
+        return PE_OK;
+      }
       // With three warps per SM the two are close; the global-state kernel loses once it has to keep the
       // per-machine records in the workspace as well (measured at V = 16384: 1.25e10 against 0.84e10
       // operator-evaluations/s at D = 8, 0.93e10 against 1.01e10 at D = 64).

@@ -30,24 +30,6 @@ namespace pe {
 constexpr int kUnroll = 8;
 constexpr uint32_t kUnscheduled = 0xFFFFFF00u;  // state words at or above this: not scheduled yet
 
-struct NarrowPtrs {
-  const uint4* ops;
-  const uint32_t* edges;
-  const int32_t* weight;
-  const uint8_t* cls;
-  const int32_t* cap;
-};
-
-__device__ __forceinline__ NarrowPtrs narrow_ptrs(const uint8_t* base, const PeNarrowView& g) {
-  NarrowPtrs p;
-  p.ops = reinterpret_cast<const uint4*>(base + g.ops);
-  p.edges = reinterpret_cast<const uint32_t*>(base + g.edges);
-  p.weight = g.has_weight ? reinterpret_cast<const int32_t*>(base + g.weight) : nullptr;
-  p.cls = base + g.cls;
-  p.cap = reinterpret_cast<const int32_t*>(base + g.cap);
-  return p;
-}
-
 // CLS: 0 = one link class, every pair connected (no table lookup); 1 = one class, some pair
 // without a channel; 2 = two classes.  IdxT: uint32_t when (V+1)*K fits in 32 bits.
 // TIMES: start and finish are both written (true) or both absent (false).

@@ -18,20 +18,26 @@
 //     delay) and sources before it (state address, delay), and finds the machine's previous
 //     operator in the window;
 //   * a baton (a named barrier between two warps) goes from window to window.  The warp that holds
-//     it gathers the end times of the sources before the window (final by then), relaxes the window
-//     with shuffles until nothing changes, publishes end << 8 | machine and passes the baton on.
-//     Only this part is serial, and it touches nothing but shared memory and registers;
+//     it gathers the end times of the sources before the window (final by then) and relaxes the window
+//     with shuffles: every lane takes the maximum over its in-window sources' current end times plus
+//     delays, for as many rounds as the window is deep (the depth is known from the set-up, so the
+//     loop needs no vote); then it publishes end << 8 | machine and passes the baton on.  Only this
+//     part is serial, it touches nothing but shared memory and registers, and it never diverges;
 //   * the memory levels follow each machine's sequence, not the times: they have their own, much
 //     shorter, baton, and run ahead of the times.
 // State word: pending = 0x80000000 | position << 8 | machine (position 0xFFFF = not in the order);
 // final = end << 8 | machine, end < 2^23.  Row V is the sentinel the compact encoding's empty edge
-// slots point at (final, end 0, machine 0).
+// slots point at (final, end 0, machine 0); row V + 1 takes the writes of lanes that have nothing to
+// write.
+//
+// Inputs and times either use the candidate-interleaved arrays of the interface directly (every lane
+// then touches its own 32-byte sector) or, STAGED, candidate-major copies made by pe_transpose_kernel,
+// where a window's order entries and times are 64 and 128 contiguous bytes.
 //
 // The kernel serves graphs in which no operator has more than three incoming edges (the inline
 // slots of the compact record are then all there is).
 #pragma once
 #include "pe_device.cuh"
-#include "pe_kernel_lane.cuh"
 
 namespace pe {
 
@@ -53,7 +59,7 @@ struct TeamStrides {
   size_t out_row, out_cand;   // start, finish
 };
 
-template <int NW, bool BY_POS, int CLS, bool TIMES, bool STAGED>
+template <int NW, bool BY_POS, int CLS, bool TIMES, bool STAGED, bool WIDE>
 __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, const uint8_t* __restrict__ nblob,
                                                                int64_t K, const uint8_t* __restrict__ assign,
                                                                const uint16_t* __restrict__ order, pe_outputs out,
@@ -266,17 +272,43 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
     // (a lane beyond the end of the order goes through the same code on operator 0's record; what it
     //  classifies and flags is dropped right after)
     const uint32_t st_before = st;
+    // WIDE: operators with four to eight incoming edges; edges 3.. take the extra slots
+    constexpr int kExtra = WIDE ? 5 : 1;
+    uint32_t xa[kExtra];
+    int32_t xg[kExtra], xd[kExtra];
+    int xl[kExtra];
+#pragma unroll
+    for (int q = 0; q < kExtra; ++q) { xa[q] = none; xg[q] = kNever; xl[q] = lane; xd[q] = kNever + dur; }
     classify(rec.z, rec.w, a0, g0, l0, d0);
     if (TWO_CLASS) {
       a1 = none; a2 = none; g1 = kNever; g2 = kNever; l1 = lane; l2 = lane; d1 = kNever + dur; d2 = kNever + dur;
       const uint2* ed = reinterpret_cast<const uint2*>(gp.edges) + rec.x;
       if (indeg > 1) { const uint2 e1 = __ldg(ed + 1); classify(e1.x, e1.y, a1, g1, l1, d1); }
       if (indeg > 2) { const uint2 e2 = __ldg(ed + 2); classify(e2.x, e2.y, a2, g2, l2, d2); }
+      if constexpr (WIDE) {
+#pragma unroll
+        for (int q = 0; q < kExtra; ++q)
+          if (indeg > 3 + q) { const uint2 eq = __ldg(ed + 3 + q); classify(eq.x, eq.y, xa[q], xg[q], xl[q], xd[q]); }
+      }
     } else {
       classify(rec.w, 0u, a1, g1, l1, d1);
-      classify(rec.x, 0u, a2, g2, l2, d2);
+      if constexpr (WIDE) {
+        // with more than three incoming edges the record's first word is the edge list's slot, not edge 2
+        const uint32_t* ed = gp.edges + rec.x;
+        const bool many = indeg > 3;
+        classify(many ? __ldg(ed + 2) : rec.x, 0u, a2, g2, l2, d2);
+#pragma unroll
+        for (int q = 0; q < kExtra; ++q)
+          if (indeg > 3 + q) classify(__ldg(ed + 3 + q), 0u, xa[q], xg[q], xl[q], xd[q]);
+      } else {
+        classify(rec.x, 0u, a2, g2, l2, d2);
+      }
     }
-    if (!act) { st = st_before; depmask = 0; a0 = a1 = a2 = none; }
+    if (!act) {
+      st = st_before; depmask = 0; a0 = a1 = a2 = none;
+#pragma unroll
+      for (int q = 0; q < kExtra; ++q) xa[q] = none;
+    }
     const int prev = 31 - __clz(below);
     const int lp = has_prev ? prev : lane;
     const int32_t dp = (has_prev ? 0 : kNever) + dur;
@@ -328,8 +360,15 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
     if (win > 0) named_sync(1 + warp, 64);
     const uint32_t w0 = state[a0], w1 = state[a1], w2 = state[a2];
     const int32_t fr = (int32_t)state[fr_at];
-    const int32_t r_base = __vimax3_s32(__viaddmax_s32((int32_t)(w0 >> 8), g0, fr), (int32_t)(w1 >> 8) + g1,
-                                        (int32_t)(w2 >> 8) + g2);
+    int32_t r_base = __vimax3_s32(__viaddmax_s32((int32_t)(w0 >> 8), g0, fr), (int32_t)(w1 >> 8) + g1,
+                                  (int32_t)(w2 >> 8) + g2);
+    if constexpr (WIDE) {
+      uint32_t xw[kExtra];
+#pragma unroll
+      for (int q = 0; q < kExtra; ++q) xw[q] = state[xa[q]];
+#pragma unroll
+      for (int q = 0; q < kExtra; ++q) r_base = __viaddmax_s32((int32_t)(xw[q] >> 8), xg[q], r_base);
+    }
     const int32_t b_end = r_base + dur;
     int32_t e = b_end;
     // every dependence points to a lower lane, so the values rise monotonically to the window's
@@ -337,7 +376,15 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
     for (int it = 0; it < nrounds; ++it) {
       const int32_t s0 = __shfl_sync(FULL, e, l0), s1 = __shfl_sync(FULL, e, l1);
       const int32_t s2 = __shfl_sync(FULL, e, l2), s3 = __shfl_sync(FULL, e, lp);
-      e = __vimax3_s32(__viaddmax_s32(s0, d0, b_end), __viaddmax_s32(s1, d1, s2 + d2), s3 + dp);
+      int32_t en = __vimax3_s32(__viaddmax_s32(s0, d0, b_end), __viaddmax_s32(s1, d1, s2 + d2), s3 + dp);
+      if constexpr (WIDE) {
+        int32_t xs[kExtra];
+#pragma unroll
+        for (int q = 0; q < kExtra; ++q) xs[q] = __shfl_sync(FULL, e, xl[q]);
+#pragma unroll
+        for (int q = 0; q < kExtra; ++q) en = __viaddmax_s32(xs[q], xd[q], en);
+      }
+      e = en;
     }
     state[st_at] = ((uint32_t)e << 8) | j;
     state[fw_at] = (uint32_t)e;

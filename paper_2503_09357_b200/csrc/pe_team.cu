@@ -30,11 +30,12 @@ int launch3(const TeamCall& t) {
                                                             t.sd);
     return PE_OK;
   };
-  if (t.p->staged)
-    return t.out.start ? go(pe_eval_team_kernel<NW, BY_POS, CLS, true, true>)
-                       : go(pe_eval_team_kernel<NW, BY_POS, CLS, false, true>);
-  return t.out.start ? go(pe_eval_team_kernel<NW, BY_POS, CLS, true, false>)
-                     : go(pe_eval_team_kernel<NW, BY_POS, CLS, false, false>);
+  const bool wide = t.g->max_indeg > 3;   // operators with four to eight incoming edges
+#define PE_TEAM(TIMES, STAGED) \
+  (wide ? go(pe_eval_team_kernel<NW, BY_POS, CLS, TIMES, STAGED, true>) : go(pe_eval_team_kernel<NW, BY_POS, CLS, TIMES, STAGED, false>))
+  if (t.p->staged) return t.out.start ? PE_TEAM(true, true) : PE_TEAM(false, true);
+  return t.out.start ? PE_TEAM(true, false) : PE_TEAM(false, false);
+#undef PE_TEAM
 }
 
 template <int NW, bool BY_POS>
