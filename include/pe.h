@@ -178,9 +178,10 @@ int pe_eval_batch_host(pe_graph* g, int64_t K, const uint8_t* host_assign, const
  * with the meaning and layouts of pe_eval_batch; flags may hold PE_ASSIGN_BY_POS and
  * PE_TIMES_BY_OP only (no variant bits).  Results are identical to pe_eval_batch's.
  *
- *  - Size limit: pe_workspace_bytes(g, K, flags | PE_VARIANT_GLOBAL) must not exceed
- *    PE_NOALLOC_SCRATCH_BYTES (about 4*V*K bytes, 5*V*K with PE_ASSIGN_BY_POS); a larger batch is
- *    refused with PE_ERR_SCRATCH_LIMIT and nothing is launched.  Split the batch instead.
+ *  - Size limit: the scratch this call's kernel needs (about 4*V*K bytes, 5*V*K with PE_ASSIGN_BY_POS
+ *    on graphs without a compact encoding; never more than pe_workspace_bytes(g, K, flags |
+ *    PE_VARIANT_GLOBAL)) must not exceed PE_NOALLOC_SCRATCH_BYTES; a larger batch is refused with
+ *    PE_ERR_SCRATCH_LIMIT and nothing is launched.  Split the batch instead.
  *  - The first call on each device looks up the array's device address (a short, synchronous
  *    set-up with that device current); make that first call before starting any stream capture.
  *  - No cudaMalloc, cudaFree or other allocating routine is called, on any call.
