@@ -238,9 +238,31 @@ static bool plan_shared(const pe_graph* g, bool allow_compact, Plan* p, bool exc
   p->compact = false;
   p->exclusive = exclusive;
   if (g->narrow_ok && allow_compact) {  // compact graph staged in shared memory next to the state
+    const size_t fixed = (size_t)g->nview.bytes + 16;
+    // 16-bit state words when the machine id and every possible end time fit together (the all-ones time
+    // field marks "not scheduled"): half the state, so twice the candidates per SM where the state is what
+    // limits them.  Blocks are multiples of 64 threads there (two warps share the words of a row).
+    int jb = 1;
+    while ((1 << jb) < g->D) ++jb;
+    if (!exclusive && jb < 16 && g->time_bound < ((int64_t)1 << (16 - jb)) - 1) {
+      const size_t per16 = (size_t)2 * (g->V + 1) + (size_t)(g->has_weight ? 20 : 16) * g->D;
+      if (fixed + 64 * per16 <= g->smem_optin) {
+        size_t T = (g->smem_optin - fixed) / per16 / 64 * 64;
+        if (T > 256) T = 256;
+        p->variant = PE_VARIANT_SHARED;
+        p->threads = (int)T;
+        p->smem = fixed + T * per16;
+        p->graph_smem = true;
+        p->workspace = 0;
+        p->ws_x_off = 0;
+        p->compact = true;
+        p->state16 = true;
+        p->jbits = jb;
+        return true;
+      }
+    }
     const size_t per = (size_t)4 * (g->V + 1) + (size_t)(g->has_weight ? 20 : 16) * g->D +
                        (exclusive ? (size_t)4 * g->D * g->D : 0);
-    const size_t fixed = (size_t)g->nview.bytes + 16;
     if (fixed + 32 * per <= g->smem_optin) {
       // A block size that is a multiple of 32 keeps every lane's state column in its own bank.  That is
       // given up only where rounding down would idle more than a sixth of the candidates that fit:

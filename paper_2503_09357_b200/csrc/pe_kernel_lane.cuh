@@ -37,15 +37,25 @@ constexpr uint32_t kUnscheduled = 0xFFFFFF00u;  // state words at or above this:
 // slots are all there is and the step is straight-line code; 0 = general (inline slots, then the list).
 // EXCL (shared-state only): channels carry one transfer at a time (PE_COMM_EXCLUSIVE; Eqs. 14-15): the end of the
 // last transfer per channel sits in shared memory as [machine pair][thread] behind the operator state.
-template <typename IdxT, bool BY_POS, int CLS, bool STATE_SMEM, bool TIMES, int DEPTH, bool EXCL = false>
+// StateT: uint32_t = end << 8 | machine; uint16_t (shared-state only) = end << jbits | machine when the graph's
+// time bound and machine count fit 16 bits together: half the shared memory per candidate, twice the
+// candidates per SM.  Two warps then share the 32-bit words of a row (one the low, one the high halves), so
+// that the 32 lanes of a warp still fall into 32 different banks.
+template <typename IdxT, bool BY_POS, int CLS, bool STATE_SMEM, bool TIMES, int DEPTH, bool EXCL = false,
+          typename StateT = uint32_t>
 __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const uint8_t* __restrict__ nblob, int64_t K,
                                                            const uint8_t* __restrict__ assign,
                                                            const uint16_t* __restrict__ order, pe_outputs out,
                                                            uint32_t flags, int* err, uint32_t* __restrict__ gstate,
-                                                           int4* __restrict__ gdev) {
+                                                           int4* __restrict__ gdev, int jbits) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   constexpr bool TWO_CLASS = CLS == 2;
   constexpr bool NEED_CLS = CLS != 0;
+  constexpr bool S16 = sizeof(StateT) == 2;
+  static_assert(!S16 || (STATE_SMEM && !EXCL), "16-bit state words: shared-state kernel without exclusive channels");
+  const uint32_t jb = S16 ? (uint32_t)jbits : 8u;                     // bits of the machine field
+  const uint32_t jmask = (1u << jb) - 1u;
+  const uint32_t unsched = S16 ? ((0xFFFFu >> jb) << jb) : kUnscheduled;   // time field all ones: not scheduled yet
   const int T = blockDim.x;
   const int t = threadIdx.x;
   const int D = g.D, V = g.V;
@@ -73,8 +83,10 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
   if (c >= K) return;
   const IdxT Ki = (IdxT)K;
   // state word of operator p is state[p * pitch]
-  uint32_t* state = STATE_SMEM ? reinterpret_cast<uint32_t*>(sm + (size_t)D * T * 16 + wsum_bytes) + t
-                               : gstate + (size_t)(c >> 5) * (size_t)(V + 1) * 32 + (c & 31);
+  // (16-bit words: thread t of the block sits at halfword 2 * (32 * (t / 64) + t % 32) + (t / 32) % 2 of a row)
+  const uint32_t t_off = S16 ? 2u * (32u * ((uint32_t)t >> 6) + ((uint32_t)t & 31u)) + (((uint32_t)t >> 5) & 1u) : (uint32_t)t;
+  StateT* state = STATE_SMEM ? reinterpret_cast<StateT*>(sm + (size_t)D * T * 16 + wsum_bytes) + t_off
+                             : reinterpret_cast<StateT*>(gstate + (size_t)(c >> 5) * (size_t)(V + 1) * 32 + (c & 31));
   const uint32_t pitch = STATE_SMEM ? (uint32_t)T : 32u;
   // EXCL: end of the last transfer on channel (j1 -> j2) at chan[(j1 * D + j2) * T]
   int32_t* chan = reinterpret_cast<int32_t*>(sm + (size_t)D * T * 16 + wsum_bytes + (size_t)(V + 1) * T * 4) + t;
@@ -82,6 +94,7 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
 
   const uint16_t* order_col = order + c;
   const uint8_t* assign_col = assign + c;
+  uint32_t raw_max = 0;   // 16-bit words, by-operator assignments: largest machine id seen before clamping
   {  // initial state: unscheduled; by-operator assignments also deposit the machine byte.  The reads of
      // `assign` go out in batches of kInitBatch so that their latency is paid once per batch, not per row.
     constexpr int kInitBatch = 16;
@@ -93,14 +106,19 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
 #pragma unroll
         for (int u = 0; u < kInitBatch; ++u) { x[u] = (uint32_t)assign_col[at]; at += Ki; }
 #pragma unroll
-        for (int u = 0; u < kInitBatch; ++u) state[(uint32_t)(i + u) * pitch] = kUnscheduled | x[u];
+        for (int u = 0; u < kInitBatch; ++u) {
+          if (S16) { raw_max = max(raw_max, x[u]); x[u] = min(x[u], (uint32_t)(D - 1)); }   // the field is only jbits wide
+          state[(uint32_t)(i + u) * pitch] = (StateT)(unsched | x[u]);
+        }
       }
     }
     for (; i < V; ++i) {
-      state[(uint32_t)i * pitch] = BY_POS ? 0xFFFFFFFFu : (kUnscheduled | (uint32_t)assign_col[at]);
+      uint32_t x1 = BY_POS ? 0u : (uint32_t)assign_col[at];
+      if (S16) { raw_max = max(raw_max, x1); x1 = min(x1, (uint32_t)(D - 1)); }
+      state[(uint32_t)i * pitch] = (StateT)(BY_POS ? 0xFFFFFFFFu : (unsched | x1));
       at += Ki;
     }
-    state[(uint32_t)V * pitch] = 0u;
+    state[(uint32_t)V * pitch] = (StateT)0;
   }
   for (int j = 0; j < D; ++j) {
     dev[j * dpitch] = make_int4(0, 0, 0, 0);
@@ -144,7 +162,7 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
     const uint32_t i = min(iu, vmax);
     const uint32_t mine = state[i * pitch];
     own_min = min(own_min, mine);
-    const uint32_t jr = BY_POS ? a_pos : (mine & 0xFFu);
+    const uint32_t jr = BY_POS ? a_pos : (mine & jmask);
     dev_max = max(dev_max, jr);
     const int j = (int)min(jr, dmax);
     const int4 dv = dev[j * dpitch];
@@ -157,7 +175,7 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
       const uint32_t p = lo & 0xFFFFu;
       const uint32_t w = state[p * pitch];
       pred_max = max(pred_max, w);
-      const int xp = (int)(w & 0xFFu);
+      const int xp = (int)(w & jmask);
       const uint32_t xpc = min((uint32_t)xp, dmax);  // (an unscheduled source of an invalid order may still carry a raw id)
       uint32_t delay = lo >> 16;
       bool channel = true;
@@ -174,13 +192,13 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
         // the transfer starts when its source has ended (Eq. 13) and the channel is free (Eq. 14), lasts D^c (Eq. 11)
         if (xp != j && p != (uint32_t)V && channel) {
           int32_t* ch = chan + (xpc * D + j) * (uint32_t)T;
-          const int32_t t_end = max((int32_t)(w >> 8), *ch) + (int32_t)delay;
+          const int32_t t_end = max((int32_t)(w >> jb), *ch) + (int32_t)delay;
           *ch = t_end;
           return t_end;
         }
-        return (int32_t)(w >> 8);
+        return (int32_t)(w >> jb);
       }
-      return (int32_t)(w >> 8) + (xp != j ? (int32_t)delay : 0);
+      return (int32_t)(w >> jb) + (xp != j ? (int32_t)delay : 0);
     };
     int32_t r = edge_time(rec.z, rec.w);
     if (TWO_CLASS) {
@@ -206,7 +224,7 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
     const int32_t e = s + dur;
     const int32_t lv = dv.z + dA;
     dev[j * dpitch] = make_int4(e, dv.y + dur, lv, max(dv.w, lv));
-    state[i * pitch] = ((uint32_t)e << 8) | (uint32_t)j;
+    state[i * pitch] = (StateT)(((uint32_t)e << jb) | (uint32_t)j);
     if (gp.weight) wsum[j * dpitch] += gp.weight[i];
     z = max(z, e);
     if (TIMES) {
@@ -231,9 +249,22 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
     if (kb + u < V) step(o0[u], a0[u], o0[(u + 1) % kUnroll]);
 
   if (order_max > vmax) st |= PE_STATUS_ORDER_INVALID;    // an entry that is no operator
-  if (own_min < kUnscheduled) st |= PE_STATUS_ORDER_INVALID;   // an operator scheduled twice
-  if (pred_max >= kUnscheduled) st |= PE_STATUS_ORDER_INVALID;  // an operator ahead of one of its predecessors
+  if (own_min < unsched) st |= PE_STATUS_ORDER_INVALID;   // an operator scheduled twice
+  if (pred_max >= unsched) st |= PE_STATUS_ORDER_INVALID;  // an operator ahead of one of its predecessors
   if (dev_max > dmax) st |= PE_STATUS_ASSIGN_RANGE;
+  if (S16 && !BY_POS && raw_max > dmax) {
+    // Some operator's machine id is out of range and was clamped when the state was set up.  The bit is due
+    // only if that operator is consulted, i.e. appears in the order: certain for a permutation, otherwise
+    // (a rare double fault) the order is walked once more.
+    if (!(st & PE_STATUS_ORDER_INVALID)) {
+      st |= PE_STATUS_ASSIGN_RANGE;
+    } else {
+      for (int k = 0; k < V; ++k) {
+        const uint32_t iu = (uint32_t)order_col[(IdxT)k * Ki];
+        if (iu <= vmax && (uint32_t)assign_col[(IdxT)iu * Ki] > dmax) st |= PE_STATUS_ASSIGN_RANGE;
+      }
+    }
+  }
   for (int j = 0; j < D; ++j) {
     const int4 dv = dev[j * dpitch];
     const int32_t pk = dv.w + (gp.weight ? wsum[j * dpitch] : 0);  // the weights are resident from the start (Eq. 16)

@@ -14,10 +14,13 @@ static int launch4(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* a
     if (p.variant == PE_VARIANT_GLOBAL && p.smem == 0)
       gdev = reinterpret_cast<int4*>(reinterpret_cast<uint8_t*>(gstate) + p.ws_x_off);
     kern<<<grid, p.threads, p.smem, stream>>>(g->nview, g->d_nblob, K, assign, order, out, flags, g->d_error, gstate,
-                                               gdev);
+                                               gdev, p.jbits);
     return PE_OK;
   };
   if constexpr (STATE_SMEM) {
+    if (p.state16)   // end time and machine fit 16 bits together: half the state per candidate
+      return out.start ? go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, true, true, DEPTH, false, uint16_t>)
+                       : go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, true, false, DEPTH, false, uint16_t>);
     if (p.exclusive)
       return out.start ? go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, true, true, DEPTH, true>)
                        : go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, true, false, DEPTH, true>);

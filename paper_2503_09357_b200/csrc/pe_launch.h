@@ -20,6 +20,8 @@ struct Plan {
   int warp_words = 0;     // WARP: 32-bit words of shared memory per candidate
   bool compact = false;   // SHARED / GLOBAL / WARP: the compact-graph kernels
   bool exclusive = false; // SHARED (compact): PE_COMM_EXCLUSIVE, one more word per machine pair and candidate
+  bool state16 = false;   // SHARED (compact): 16-bit state words, end << jbits | machine
+  int jbits = 8;          // bits of the machine field of a state word
   bool slab = false;      // WARP (compact): order entries and times go through shared tiles, a slab at a time
   // TEAM: inputs and times go through candidate-major staging copies in the workspace, a chunk of candidates at a time
   bool staged = false;
