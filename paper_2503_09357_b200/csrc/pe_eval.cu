@@ -742,8 +742,9 @@ extern "C" int pe_eval_batch_noalloc(pe_graph* g, int64_t K, const uint8_t* assi
   if (ret == PE_OK) {
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const bool by_pos = (flags & PE_ASSIGN_BY_POS) != 0;
-    // launch_typed clears the end-time state (the part of the scratch that must start as "not
-    // scheduled") on the stream before the kernel, so the previous call's contents never matter
+    // whatever the previous call left in the array never matters: the generic kernel's end times are
+    // cleared by a memset that launch_typed puts on the stream before the kernel, and the compact kernel
+    // writes every state word ("not scheduled") and per-machine record itself before it reads any
     if (order_bytes == 2)
       ret = by_pos ? pe::launch_typed<uint16_t, true>(g, p, K, assign, order, flags, *out, scratch, stream)
                    : pe::launch_typed<uint16_t, false>(g, p, K, assign, order, flags, *out, scratch, stream);

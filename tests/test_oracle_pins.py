@@ -43,8 +43,6 @@ TINY = [
 @pytest.mark.parametrize("D", [1, 2, 3])
 def test_exhaustive_candidates_satisfy_constraints_and_are_left_shifted(case, D):
     V, edges, dur, comm = TINY[case]
-    if D == 3 and V == 5:
-        pytest.skip("kept small")
     A = [((3 * i) % 5) - 2 for i in range(V)]
     w = ck.problem(V, edges, dur, D, comm=np.array(comm, np.int32).reshape(-1, 1) if comm else None, A=A)
     xs, pis = [], []

@@ -493,3 +493,62 @@ def test_many_sources_of_one_operator_inside_its_window(pe):
         gu.check(g, w, a_pos, order, flags=pe.PE_VARIANT_WARP | pe.PE_ASSIGN_BY_POS, label="many in-window sources by-pos")
     finally:
         g.close()
+
+
+@pytest.mark.parametrize("K", [333, 332])
+def test_team_kernel_with_and_without_staging_copies(pe, K):
+    """The block-per-candidate kernel reads the interleaved arrays directly when K is not a multiple of 4 (K = 333)
+    and goes through candidate-major staging copies otherwise (K = 332); both, in every layout, on a graph large
+    enough for it to be the automatic choice, and on the MoE graph (operators with eight incoming edges)."""
+    for w in (wl.make_config(5, V=4096, D=8), wl.make_config(3)):
+        assign, order = wl.make_candidates(w, K=K)
+        g = pe.Graph(w)
+        try:
+            assert g.variant(K) == "team"
+            for base in (0, pe.PE_ASSIGN_BY_POS, pe.PE_TIMES_BY_OP, pe.PE_ASSIGN_BY_POS | pe.PE_TIMES_BY_OP):
+                a = wl.assign_by_pos(assign, order) if base & pe.PE_ASSIGN_BY_POS else assign
+                gu.check(g, w, a, order, flags=base | pe.PE_VARIANT_TEAM, label=f"team K={K} flags={base}")
+            gu.check(g, w, assign, order, flags=pe.PE_VARIANT_TEAM, want_times=False, label=f"team K={K} summary")
+        finally:
+            g.close()
+
+
+def test_two_host_threads_share_a_graph(pe):
+    """pe.h promises that a graph may be used from several host threads and streams.  The block-per-candidate
+    variant forks onto side streams owned by the graph, so two threads, each with its own stream, workspace and
+    outputs, evaluate different batches at the same time, several times over; both must get the oracle's result."""
+    import threading
+    import torch
+    from oracle import pe_oracle as orc
+    w = wl.make_config(5, V=4096, D=64)
+    K = 8000                                                   # more than one chunk: the side streams are used
+    g = pe.Graph(w)
+    try:
+        batches = [wl.make_candidates(w, K=K, first=n * K) for n in range(2)]
+        refs = [orc.evaluate(w, a, o, threads=gu.CPU_THREADS) for a, o in batches]
+        errors = []
+
+        def work(n):
+            try:
+                a, o = batches[n]
+                s = torch.cuda.Stream()
+                with torch.cuda.stream(s):
+                    da = torch.from_numpy(a).cuda(); do = torch.from_numpy(gu.as_signed(o)).cuda()
+                    ws = g.alloc_workspace(K, 0)
+                    for _ in range(4):
+                        out = g.eval_batch(da, do, workspace=ws, stream=s.cuda_stream)
+                    s.synchronize()
+                res = {k: v.cpu().numpy() for k, v in out.items()}
+                res["status"] = res["status"].view(np.uint32)
+                gu.compare(res, refs[n], f"thread {n}")
+            except Exception as e:                               # reported by the main thread
+                errors.append(e)
+
+        threads = [threading.Thread(target=work, args=(n,)) for n in range(2)]
+        for t in threads:
+            t.start()
+        for t in threads:
+            t.join()
+        assert not errors, errors
+    finally:
+        g.close()
