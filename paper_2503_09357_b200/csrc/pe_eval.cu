@@ -385,8 +385,9 @@ static bool plan_team(const pe_graph* g, int64_t K, bool allow_compact, Plan* p)
 
 static bool plan_global(const pe_graph* g, int64_t K, uint32_t flags, bool allow_compact, Plan* p) {
   p->compact = false;
-  const bool exclusive = (flags & PE_COMM_EXCLUSIVE) != 0;   // only the generic kernel sequences transfers per channel
-  if (!exclusive && g->narrow_ok && allow_compact && g->time_bound < kPackedTimeLimit) {
+  const bool exclusive = (flags & PE_COMM_EXCLUSIVE) != 0;
+  p->exclusive = exclusive;
+  if (g->narrow_ok && allow_compact && g->time_bound < kPackedTimeLimit) {
     // compact-graph kernel with the state in the workspace.  Per-machine records stay in shared
     // memory while a 128-thread block needs at most 16 KB for them; beyond that they would cap the
     // resident candidates, so they move to the workspace too (tiles that stay in L2).
@@ -406,6 +407,8 @@ static bool plan_global(const pe_graph* g, int64_t K, uint32_t flags, bool allow
       p->ws_x_off = state_bytes;  // offset of the per-machine records
       p->workspace = state_bytes + round_up(tiles * 32 * per, 256);
     }
+    p->ws_c_off = p->workspace;   // PE_COMM_EXCLUSIVE: end of the last transfer per channel, tiles [tile][D*D][32]
+    if (exclusive) p->workspace += round_up(tiles * 32 * (size_t)g->D * g->D * 4, 256);
     return true;
   }
   const size_t per_thread = (size_t)20 * g->D;

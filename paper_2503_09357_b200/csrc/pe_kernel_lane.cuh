@@ -35,8 +35,9 @@ constexpr uint32_t kUnscheduled = 0xFFFFFF00u;  // state words at or above this:
 // TIMES: start and finish are both written (true) or both absent (false).
 // DEPTH (one link class only): 3 = no operator has more than three incoming edges, so the three inline
 // slots are all there is and the step is straight-line code; 0 = general (inline slots, then the list).
-// EXCL (shared-state only): channels carry one transfer at a time (PE_COMM_EXCLUSIVE; Eqs. 14-15): the end of the
-// last transfer per channel sits in shared memory as [machine pair][thread] behind the operator state.
+// EXCL: channels carry one transfer at a time (PE_COMM_EXCLUSIVE; Eqs. 14-15): the end of the last transfer per
+// channel sits in shared memory as [machine pair][thread] behind the operator state (shared-state kernel) or in the
+// workspace as tiles [tile of 32][machine pair][32] behind everything else (global-state kernel).
 // StateT: uint32_t = end << 8 | machine; uint16_t (shared-state only) = end << jbits | machine when the graph's
 // time bound and machine count fit 16 bits together: half the shared memory per candidate, twice the
 // candidates per SM.  Two warps then share the 32-bit words of a row (one the low, one the high halves), so
@@ -47,7 +48,8 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
                                                            const uint8_t* __restrict__ assign,
                                                            const uint16_t* __restrict__ order, pe_outputs out,
                                                            uint32_t flags, int* err, uint32_t* __restrict__ gstate,
-                                                           int4* __restrict__ gdev, int jbits) {
+                                                           int4* __restrict__ gdev, int jbits,
+                                                           int32_t* __restrict__ gchan) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   constexpr bool TWO_CLASS = CLS == 2;
   constexpr bool NEED_CLS = CLS != 0;
@@ -88,9 +90,11 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
   StateT* state = STATE_SMEM ? reinterpret_cast<StateT*>(sm + (size_t)D * T * 16 + wsum_bytes) + t_off
                              : reinterpret_cast<StateT*>(gstate + (size_t)(c >> 5) * (size_t)(V + 1) * 32 + (c & 31));
   const uint32_t pitch = STATE_SMEM ? (uint32_t)T : 32u;
-  // EXCL: end of the last transfer on channel (j1 -> j2) at chan[(j1 * D + j2) * T]
-  int32_t* chan = reinterpret_cast<int32_t*>(sm + (size_t)D * T * 16 + wsum_bytes + (size_t)(V + 1) * T * 4) + t;
-  static_assert(!EXCL || STATE_SMEM, "exclusive channels are kept in shared memory");
+  // EXCL: end of the last transfer on channel (j1 -> j2) at chan[(j1 * D + j2) * cpitch]
+  const uint32_t cpitch = STATE_SMEM ? (uint32_t)T : 32u;
+  int32_t* chan = STATE_SMEM
+                      ? reinterpret_cast<int32_t*>(sm + (size_t)D * T * 16 + wsum_bytes + (size_t)(V + 1) * T * 4) + t
+                      : gchan + (size_t)(c >> 5) * (size_t)D * (size_t)D * 32 + (c & 31);
 
   const uint16_t* order_col = order + c;
   const uint8_t* assign_col = assign + c;
@@ -125,7 +129,7 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
     if (gp.weight) wsum[j * dpitch] = 0;
   }
   if (EXCL)
-    for (int q = 0; q < D * D; ++q) chan[(uint32_t)q * (uint32_t)T] = 0;
+    for (int q = 0; q < D * D; ++q) chan[(uint32_t)q * cpitch] = 0;
   const bool by_op_times = (flags & PE_TIMES_BY_OP) != 0;
   const bool deep = g.max_indeg > 2;
   const uint32_t vmax = (uint32_t)(V - 1), dmax = (uint32_t)(D - 1);
@@ -191,7 +195,7 @@ __global__ void __launch_bounds__(256) pe_eval_lane_kernel(PeNarrowView g, const
       if (EXCL) {
         // the transfer starts when its source has ended (Eq. 13) and the channel is free (Eq. 14), lasts D^c (Eq. 11)
         if (xp != j && p != (uint32_t)V && channel) {
-          int32_t* ch = chan + (xpc * D + j) * (uint32_t)T;
+          int32_t* ch = chan + (xpc * D + j) * cpitch;
           const int32_t t_end = max((int32_t)(w >> jb), *ch) + (int32_t)delay;
           *ch = t_end;
           return t_end;

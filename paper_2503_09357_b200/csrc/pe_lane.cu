@@ -13,8 +13,11 @@ static int launch4(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* a
     int4* gdev = nullptr;
     if (p.variant == PE_VARIANT_GLOBAL && p.smem == 0)
       gdev = reinterpret_cast<int4*>(reinterpret_cast<uint8_t*>(gstate) + p.ws_x_off);
+    int32_t* gchan = nullptr;   // GLOBAL with exclusive channels: the per-channel words follow everything else
+    if (p.variant == PE_VARIANT_GLOBAL && p.exclusive)
+      gchan = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(gstate) + p.ws_c_off);
     kern<<<grid, p.threads, p.smem, stream>>>(g->nview, g->d_nblob, K, assign, order, out, flags, g->d_error, gstate,
-                                               gdev, p.jbits);
+                                               gdev, p.jbits, gchan);
     return PE_OK;
   };
   if constexpr (STATE_SMEM) {
@@ -24,6 +27,11 @@ static int launch4(const pe_graph* g, const Plan& p, int64_t K, const uint8_t* a
     if (p.exclusive)
       return out.start ? go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, true, true, DEPTH, true>)
                        : go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, true, false, DEPTH, true>);
+  }
+  if constexpr (!STATE_SMEM) {
+    if (p.exclusive)
+      return out.start ? go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, false, true, DEPTH, true>)
+                       : go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, false, false, DEPTH, true>);
   }
   return out.start ? go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, true, DEPTH>)
                    : go(pe_eval_lane_kernel<IdxT, BY_POS, CLS, STATE_SMEM, false, DEPTH>);
