@@ -351,10 +351,16 @@ static bool plan_team(const pe_graph* g, int64_t K, bool allow_compact, Plan* p)
   if (!g->narrow_ok || !allow_compact || g->max_indeg > 8 || g->time_bound >= (int64_t)1 << 23) return false;
   const size_t smem = round_up((size_t)4 * (g->V + 2) + (size_t)4 * (5 * g->D + 2), 16);
   if (smem > g->smem_optin) return false;
-  // blocks an SM holds by shared memory; six warps per block unless that would run into the SM's thread limit
+  // Blocks an SM holds by shared memory decide the warps per block.  Few large blocks: six warps, so that the
+  // set-up of five windows hides behind the serial part of one.  Many small blocks: two warps each - a block
+  // reserves two named barriers per warp, an SM has 64 of them, and more chains beat deeper pipelines there
+  // (measured at V = 4096 / D = 64: 4.46e10 with two warps, 4.36e10 with four, 3.3e10 with six; the MoE graph:
+  // 2.03e10 against 1.96e10 and 1.63e10).
   size_t per_sm = (g->smem_per_sm ? g->smem_per_sm : g->smem_optin) / (smem + 1024);
   if (per_sm < 1) per_sm = 1;
-  const int nw = per_sm * 6 * 32 <= 2048 ? 6 : 4;
+  const int nw = per_sm <= 4 ? 6 : (per_sm <= 7 ? 4 : 2);
+  const size_t by_barriers = (size_t)64 / (nw == 6 ? 16 : 2 * nw + 1);
+  if (per_sm > by_barriers) per_sm = by_barriers;
   if (per_sm * nw * 32 > 2048) per_sm = 2048 / (nw * 32);
   p->variant = PE_VARIANT_TEAM;
   p->threads = 32 * nw;

@@ -44,12 +44,47 @@ namespace pe {
 constexpr uint32_t kTeamPending = 0x80000000u;
 constexpr int64_t kTeamTimeLimit = (int64_t)1 << 23;   // end times must stay below this
 
-// Named barriers: `count` threads in all; the warps that call named_arrive do not wait.
-__device__ __forceinline__ void named_sync(int id, int count) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+// Named barriers between pairs of warps (64 threads: the warp that arrives does not wait).  The barrier
+// numbers are immediates selected by a switch on the warp index: with a register operand the compiler
+// reserves all sixteen barriers of a block, and an SM has barrier resources for only four such blocks.
+template <int ID>
+__device__ __forceinline__ void bar_sync_id() {
+  asm volatile("bar.sync %0, 64;" ::"n"(ID) : "memory");
 }
-__device__ __forceinline__ void named_arrive(int id, int count) {
-  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+template <int ID>
+__device__ __forceinline__ void bar_arrive_id() {
+  asm volatile("bar.arrive %0, 64;" ::"n"(ID) : "memory");
+}
+// barrier number = BASE + w, w in 0 .. NW - 1 (warp-uniform).  IMM: a row of one-instruction conditionals on
+// immediates (the comparisons are loop invariant: NW predicated instructions, no branch); otherwise one
+// instruction with the number in a register, which is faster under the baton (measured at V = 16384 with six
+// warps: 16.2 against 18.8 ms for 32768 candidates) and is used where shared memory allows no more than four
+// blocks per SM anyway.
+template <int BASE, int NW, bool IMM>
+__device__ __forceinline__ void named_sync(int w) {
+  if (!IMM) {
+    asm volatile("bar.sync %0, 64;" ::"r"(BASE + w) : "memory");
+    return;
+  }
+  if (w == 0) bar_sync_id<BASE + 0>();
+  if (w == 1) bar_sync_id<BASE + 1>();
+  if (NW > 2 && w == 2) bar_sync_id<BASE + 2>();
+  if (NW > 3 && w == 3) bar_sync_id<BASE + 3>();
+  if (NW > 4 && w == 4) bar_sync_id<BASE + 4>();
+  if (NW > 5 && w == 5) bar_sync_id<BASE + 5>();
+}
+template <int BASE, int NW, bool IMM>
+__device__ __forceinline__ void named_arrive(int w) {
+  if (!IMM) {
+    asm volatile("bar.arrive %0, 64;" ::"r"(BASE + w) : "memory");
+    return;
+  }
+  if (w == 0) bar_arrive_id<BASE + 0>();
+  if (w == 1) bar_arrive_id<BASE + 1>();
+  if (NW > 2 && w == 2) bar_arrive_id<BASE + 2>();
+  if (NW > 3 && w == 3) bar_arrive_id<BASE + 3>();
+  if (NW > 4 && w == 4) bar_arrive_id<BASE + 4>();
+  if (NW > 5 && w == 5) bar_arrive_id<BASE + 5>();
 }
 
 // Element (row, c) of an input or output array sits at row * row_stride + c * cand_stride: (K, 1) for
@@ -65,11 +100,12 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
                                                                const uint16_t* __restrict__ order, pe_outputs out,
                                                                uint32_t flags, TeamStrides sd) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  static_assert(2 * NW + 1 <= 16, "two named barriers per warp, barrier 0 is the block's");
+  static_assert(NW >= 2 && NW <= 6, "two named barriers per warp (numbers 1 .. 2 NW), barrier 0 is the block's");
   constexpr uint32_t FULL = 0xFFFFFFFFu;
   constexpr bool TWO_CLASS = CLS == 2;
   constexpr bool NEED_CLS = CLS != 0;
   constexpr int NT = NW * 32;
+  constexpr bool IMMBAR = NW < 6;   // six warps per block go with large states, where few blocks fit anyway
   constexpr int32_t kNever = -(1 << 29);   // delay of an empty slot: never wins the maximum
   const int tid = threadIdx.x;
   const int lane = tid & 31;
@@ -341,7 +377,7 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
       atomicAdd(&busy[j], dur);
       if (gp.weight) atomicAdd(&wsum[j], gp.weight[i]);
     }
-    if (win > 0) named_sync(1 + NW + warp, 64);
+    if (win > 0) named_sync<1 + NW, NW, IMMBAR>(warp);
     if (act) {
       lv += lvl[j];
       atomicMax(&peak[j], lv);
@@ -349,7 +385,7 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
     __syncwarp();
     if (act && last_on_dev) lvl[j] = lv;
     __syncwarp();
-    if (win + 1 < nwin) named_arrive(1 + NW + next_warp, 64);
+    if (win + 1 < nwin) named_arrive<1 + NW, NW, IMMBAR>(next_warp);
 
     // ---- times, under the baton: every earlier window is final ----
     // (all accesses under the baton are unconditional: a lane with nothing to read reads the sentinel,
@@ -357,7 +393,7 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
     const uint32_t fr_at = (act && !has_prev) ? (uint32_t)(V + 2) + j : none;            // machine free since
     const uint32_t st_at = act ? i : none + 1u;                                           // own state word
     const uint32_t fw_at = (act && last_on_dev) ? (uint32_t)(V + 2) + j : none + 1u;      // machine free from
-    if (win > 0) named_sync(1 + warp, 64);
+    if (win > 0) named_sync<1, NW, IMMBAR>(warp);
     const uint32_t w0 = state[a0], w1 = state[a1], w2 = state[a2];
     const int32_t fr = (int32_t)state[fr_at];
     int32_t r_base = __vimax3_s32(__viaddmax_s32((int32_t)(w0 >> 8), g0, fr), (int32_t)(w1 >> 8) + g1,
@@ -389,7 +425,7 @@ __global__ void __launch_bounds__(NW * 32) pe_eval_team_kernel(PeNarrowView g, c
     state[st_at] = ((uint32_t)e << 8) | j;
     state[fw_at] = (uint32_t)e;
     __syncwarp();
-    if (win + 1 < nwin) named_arrive(1 + next_warp, 64);
+    if (win + 1 < nwin) named_arrive<1, NW, IMMBAR>(next_warp);
 
     // ---- after the baton has gone: outputs ----
     z = max(z, e);

@@ -26,6 +26,9 @@ template <int NW, bool BY_POS, int CLS>
 int launch3(const TeamCall& t) {
   auto go = [&](auto kern) -> int {
     if (!set_smem(kern, t.p->smem)) return PE_ERR_CUDA;
+    // the state is all these blocks need from the SM's memory: ask for the largest shared-memory carve-out
+    // (a hint; without it the default carve-out can hold fewer blocks than shared memory would allow)
+    cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
     kern<<<(unsigned)t.kc, NW * 32, t.p->smem, t.stream>>>(t.g->nview, t.g->d_nblob, t.K, t.assign, t.order, t.out, t.flags,
                                                             t.sd);
     return PE_OK;
@@ -49,6 +52,7 @@ int launch2(const TeamCall& t) {
 template <bool BY_POS>
 int launch1(const TeamCall& t) {
   switch (t.p->threads / 32) {
+    case 2: return launch2<2, BY_POS>(t);
     case 4: return launch2<4, BY_POS>(t);
     case 6: return launch2<6, BY_POS>(t);
     default: return PE_ERR_UNSUPPORTED;
