@@ -44,14 +44,14 @@ KERNEL_OF_VARIANT = {"shared": "pe_eval_lane_kernel<STATE_SMEM=true>", "global":
 # from an ncu capture, keyed by kernel variant, valid only while the sources that kernel is built from hash to
 # the value recorded with it.  Reported as null when those sources have changed since the capture.
 KERNEL_SOURCES = {
-    "team": ("pe_kernel_team.cuh", "pe_team.cu", "pe_transpose.cuh"),
-    "warp": ("pe_kernel_warp2.cuh", "pe_warp2.cu", "pe_device.cuh", "pe_kernel_lane.cuh"),
-    "global": ("pe_kernel_lane.cuh", "pe_lane.cu", "pe_device.cuh"),
-    "shared": ("pe_kernel_lane.cuh", "pe_lane.cu", "pe_device.cuh"),
+    "team": ("pe_kernel_team.cuh", "pe_team.cu", "pe_team_launch.h", "pe_transpose.cuh"),
+    "warp": ("pe_kernel_warp2.cuh", "pe_warp2_launch.h", "pe_device.cuh", "pe_kernel_lane.cuh"),
+    "global": ("pe_kernel_lane.cuh", "pe_lane_launch.h", "pe_device.cuh"),
+    "shared": ("pe_kernel_lane.cuh", "pe_lane_launch.h", "pe_device.cuh"),
 }
 NCU_TRAFFIC = {
     # variant: (hash of its sources at capture time, DRAM bytes per operator-evaluation, captured workload)
-    "team": ("3e8ac735e4874af7", 10.13, "random_layered_V16384_D64 at K = 3552 (one chunk), scaled by operator-evaluations; "
+    "team": ("4666c67cc9d284d0", 10.13, "random_layered_V16384_D64 at K = 3552 (one chunk), scaled by operator-evaluations; "
                         "the staging transpositions around the kernel move another 22 B per operator-evaluation"),
 }
 

@@ -7,7 +7,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libpe.so")
-SOURCES = ["pe_graph.cu", "pe_eval.cu", "pe_lane.cu", "pe_warp2.cu", "pe_team.cu", "pe_select.cu", "pe_decode.cu", "pe_coarsen.cu"]
+SOURCES = ["pe_graph.cu", "pe_eval.cu", "pe_lane.cu", "pe_lane_op.cu", "pe_lane_pos.cu", "pe_warp2.cu", "pe_warp2_op.cu", "pe_warp2_pos.cu", "pe_team.cu", "pe_team_nw2.cu", "pe_team_nw4.cu", "pe_team_nw6.cu", "pe_select.cu", "pe_decode.cu", "pe_coarsen.cu"]
 OBJ_DIR = os.path.join(_HERE, "_build")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--compiler-options", "-fPIC", "-cudart", "shared"]

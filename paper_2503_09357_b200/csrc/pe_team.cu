@@ -1,6 +1,5 @@
-// Instantiations and launcher of pe_eval_team_kernel, with the staging transpositions around it.
-#include "pe_kernel_team.cuh"
-#include "pe_launch.h"
+// Launcher of pe_eval_team_kernel (instantiated in pe_team_nw*.cu), with the staging transpositions around it.
+#include "pe_team_launch.h"
 #include "pe_transpose.cuh"
 
 #include <mutex>
@@ -9,52 +8,12 @@ namespace pe {
 
 namespace {
 
-struct TeamCall {
-  const pe_graph* g;
-  const Plan* p;
-  int64_t K;        // row pitch of the interface arrays
-  int64_t kc;       // candidates of this launch
-  const uint8_t* assign;
-  const uint16_t* order;
-  uint32_t flags;
-  pe_outputs out;
-  TeamStrides sd;
-  cudaStream_t stream;
-};
-
-template <int NW, bool BY_POS, int CLS>
-int launch3(const TeamCall& t) {
-  auto go = [&](auto kern) -> int {
-    if (!set_smem(kern, t.p->smem)) return PE_ERR_CUDA;
-    // the state is all these blocks need from the SM's memory: ask for the largest shared-memory carve-out
-    // (a hint; without it the default carve-out can hold fewer blocks than shared memory would allow)
-    cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
-    kern<<<(unsigned)t.kc, NW * 32, t.p->smem, t.stream>>>(t.g->nview, t.g->d_nblob, t.K, t.assign, t.order, t.out, t.flags,
-                                                            t.sd);
-    return PE_OK;
-  };
-  const bool wide = t.g->max_indeg > 3;   // operators with four to eight incoming edges
-#define PE_TEAM(TIMES, STAGED) \
-  (wide ? go(pe_eval_team_kernel<NW, BY_POS, CLS, TIMES, STAGED, true>) : go(pe_eval_team_kernel<NW, BY_POS, CLS, TIMES, STAGED, false>))
-  if (t.p->staged) return t.out.start ? PE_TEAM(true, true) : PE_TEAM(false, true);
-  return t.out.start ? PE_TEAM(true, false) : PE_TEAM(false, false);
-#undef PE_TEAM
-}
-
-template <int NW, bool BY_POS>
-int launch2(const TeamCall& t) {
-  const int cls = t.g->nview.L == 2 ? 2 : (t.g->nview.need_cls ? 1 : 0);
-  if (cls == 2) return launch3<NW, BY_POS, 2>(t);
-  if (cls == 1) return launch3<NW, BY_POS, 1>(t);
-  return launch3<NW, BY_POS, 0>(t);
-}
-
 template <bool BY_POS>
 int launch1(const TeamCall& t) {
   switch (t.p->threads / 32) {
-    case 2: return launch2<2, BY_POS>(t);
-    case 4: return launch2<4, BY_POS>(t);
-    case 6: return launch2<6, BY_POS>(t);
+    case 2: return launch_team_nw2(t, BY_POS);
+    case 4: return launch_team_nw4(t, BY_POS);
+    case 6: return launch_team_nw6(t, BY_POS);
     default: return PE_ERR_UNSUPPORTED;
   }
 }
