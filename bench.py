@@ -51,7 +51,7 @@ KERNEL_SOURCES = {
 }
 NCU_TRAFFIC = {
     # variant: (hash of its sources at capture time, DRAM bytes per operator-evaluation, captured workload)
-    "team": ("4666c67cc9d284d0", 10.13, "random_layered_V16384_D64 at K = 3552 (one chunk), scaled by operator-evaluations; "
+    "team": ("698c9fc757a7e542", 10.13, "random_layered_V16384_D64 at K = 3552 (one chunk), scaled by operator-evaluations; "
                         "the staging transpositions around the kernel move another 22 B per operator-evaluation"),
 }
 

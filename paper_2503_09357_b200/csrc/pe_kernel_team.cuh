@@ -34,8 +34,8 @@
 // then touches its own 32-byte sector) or, STAGED, candidate-major copies made by pe_transpose_kernel,
 // where a window's order entries and times are 64 and 128 contiguous bytes.
 //
-// The kernel serves graphs in which no operator has more than three incoming edges (the inline
-// slots of the compact record are then all there is).
+// The kernel serves graphs in which no operator has more than eight incoming edges: three slots for the
+// edges the compact record carries inline, and (WIDE) five more for edges read from the edge list.
 #pragma once
 #include "pe_device.cuh"
 
@@ -44,9 +44,9 @@ namespace pe {
 constexpr uint32_t kTeamPending = 0x80000000u;
 constexpr int64_t kTeamTimeLimit = (int64_t)1 << 23;   // end times must stay below this
 
-// Named barriers between pairs of warps (64 threads: the warp that arrives does not wait).  The barrier
-// numbers are immediates selected by a switch on the warp index: with a register operand the compiler
-// reserves all sixteen barriers of a block, and an SM has barrier resources for only four such blocks.
+// Named barriers between pairs of warps (64 threads: the warp that arrives does not wait).  With the barrier
+// number in a register the compiler reserves all sixteen barriers of a block, and an SM has barrier resources
+// for only four such blocks; with immediates it reserves what is used (two per warp plus the block's own).
 template <int ID>
 __device__ __forceinline__ void bar_sync_id() {
   asm volatile("bar.sync %0, 64;" ::"n"(ID) : "memory");
